@@ -1,0 +1,152 @@
+/*
+ * dkv.h -- C ABI of libdkv: DynamicKV prefill-time KV-cache compression on one NVIDIA B200.
+ *
+ * The library implements the data-parallel path of Algorithm 1 ("DynamicKV in Prefill Phase",
+ * arXiv 2412.14838): per layer, score every prefix token against the observation-window
+ * queries (Eq. 1-2), keep the per-layer maximum budget B^l per head (Eq. 3), every m layers
+ * re-derive the per-layer counts from a global top-K over all accumulated scores (Eq. 4-6),
+ * and shrink the buffers of all preceding layers to those counts.
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, 16-byte aligned, contiguous in
+ *     the stated layout, unless the argument is documented as a host pointer.  The library never
+ *     frees or reallocates caller memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls enqueue
+ *     work and return; only dkv_create, dkv_destroy, dkv_get_counts, dkv_last_status and
+ *     dkv_run_prefill_pass_host synchronise.
+ *   - A context belongs to one device (the one current at dkv_create) and to one stream at a time.
+ *   - Return value: 0 = DKV_OK, negative = error (below).  Nothing is printed, nothing aborts.
+ *   - Layer numbers are 0-based.  Algorithm 1's test "l % m == 0" uses 1-based l, i.e. an update
+ *     follows API layers m-1, 2m-1, ...
+ *   - Shapes: L layers, Hq query heads, Hkv KV heads (G = Hq/Hkv), D head size, Bt samples, S prompt
+ *     length including the window, ws window, P = S - ws prefix tokens, N = wt - ws average budget,
+ *     Bl = B^l = N * r_max per-layer maximum, Bl' = min(Bl, P).
+ *   - bf16 tensors are raw 16-bit patterns.  Samples of a batch are independent problems.
+ */
+#ifndef DKV_H_
+#define DKV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DKV_OK                 0
+#define DKV_ERR_INVALID_ARG   -1   /* NULL/misaligned pointer, value out of range                  */
+#define DKV_ERR_STATE         -2   /* call order: e.g. select before score                         */
+#define DKV_ERR_CUDA          -3   /* a CUDA runtime call failed (dkv_last_cuda_error has the code) */
+#define DKV_ERR_TIMEOUT       -4   /* a bounded device-side wait ran out                           */
+#define DKV_ERR_UNSUPPORTED   -5   /* shape outside the compiled set                               */
+#define DKV_ERR_NOMEM         -6   /* device or host allocation failed                             */
+
+#define DKV_MAX_LAYERS        128
+#define DKV_MAX_LAYER_BUDGET  16384  /* Bl  */
+#define DKV_MAX_WINDOW_ROWS   256    /* ws * G */
+
+typedef struct dkv_ctx dkv_ctx;     /* opaque; owns score history, kept indices, ranks, counts, workspace */
+
+/* Problem statement of Algorithm 1 (its inputs r_max, m, wt, ws, S, d_k) plus the model shape. */
+typedef struct {
+  int32_t n_layers;         /* L   : 1..DKV_MAX_LAYERS                                            */
+  int32_t n_q_heads;        /* Hq  : multiple of n_kv_heads                                       */
+  int32_t n_kv_heads;       /* Hkv                                                                */
+  int32_t head_dim;         /* D   : 64 or 128                                                    */
+  int32_t batch;            /* Bt                                                                 */
+  int32_t seq_len;          /* S   : includes the window; S > ws                                  */
+  int32_t window;           /* ws  : ws * G <= DKV_MAX_WINDOW_ROWS                                */
+  int32_t pool_kernel;      /* odd width of the 1-D pooling of Eq. 2, >= 1                        */
+  int32_t pool_kind;        /* 0 = max-pool (only kind built)                                     */
+  int32_t avg_budget;       /* N = wt - ws : retained prefix tokens per head per layer on average */
+  int32_t layer_max;        /* Bl = floor(N * r_max), N <= Bl <= DKV_MAX_LAYER_BUDGET             */
+  int32_t update_interval;  /* m >= 1                                                             */
+  uint32_t flags;           /* must be 0                                                          */
+} dkv_config;
+
+/* Create a context for `cfg` on the current device (host call; allocates device memory:
+ * score history 4*L*Bt*Hkv*P bytes, kept indices and ranks 8*L*Bt*Hkv*Bl' bytes, small workspaces).
+ * Errors: INVALID_ARG, UNSUPPORTED, NOMEM, CUDA.  On error *out is NULL. */
+int dkv_create(const dkv_config* cfg, dkv_ctx** out);
+/* Free everything the context owns (synchronises the device). */
+int dkv_destroy(dkv_ctx* ctx);
+/* Forget all layers: a new prompt.  Enqueued on `stream`. */
+int dkv_reset(dkv_ctx* ctx, void* stream);
+
+/* (1) Eq. 1-2 / Algorithm 1 scoring line.  For every sample b, KV head h and prefix position j < P:
+ *       raw[j]   = sum over the G query heads of the group and the ws window rows r of
+ *                  softmax_row(q . K^T / sqrt(D))[j], row r's softmax running over keys 0 .. P+r;
+ *       score[j] = max of raw over |j' - j| <= pool_kernel/2, 0 <= j' < P.
+ *     q_win : bf16 [Bt, Hq, ws, D]   queries of the last ws positions
+ *     k     : bf16 [Bt, Hkv, S, D]   keys of the layer
+ *     scores_out : fp32 [Bt, Hkv, P] optional copy of the result (NULL = keep it in the context only)
+ *     bf16 inputs, fp32 accumulation.  Stores the scores as layer `layer` of the context's history. */
+int dkv_score(dkv_ctx* ctx, int32_t layer, const void* q_win, const void* k, float* scores_out, void* stream);
+
+/* Store caller-computed scores fp32 [Bt, Hkv, P] (finite, >= 0) as layer `layer` of the history,
+ * in place of dkv_score (e.g. scores emitted by a fused prefill attention kernel). */
+int dkv_set_scores(dkv_ctx* ctx, int32_t layer, const float* scores, void* stream);
+
+/* (2) Eq. 3 / Algorithm 1 "topk(B^l)".  Per (b, h): the Bl' positions with the largest score under the
+ *     total order (score descending, position ascending).
+ *     idx_out  : int32 [Bt, Hkv, Bl'] kept positions, ascending (optional)
+ *     rank_out : int32 [Bt, Hkv, Bl'] place of each kept position in the total order, 0 = best (optional)
+ *     Sets count[b][layer] = Bl'.  Needs the layer's scores (else DKV_ERR_STATE). */
+int dkv_select_topk(dkv_ctx* ctx, int32_t layer, int32_t* idx_out, int32_t* rank_out, void* stream);
+
+/* (3) Eq. 4-6 / Update_Buffer_Length after `upto_layer` layers (1..L; all of them scored and selected).
+ *     Per sample: k = min(N*Hkv*l, l*Hkv*P) largest history scores of layers [0, l), ties to the lowest
+ *     flat index (layer, head, position); cnt_i = hits in layer i; Z_i = floor(Bl*cnt_i / max cnt);
+ *     Z'_i = floor(Z_i * N*L / sum Z); count[b][i] = min(count[b][i], Z'_i).  All on the device.
+ *     counts_out : int32 [Bt, L] device copy of the counts after the update (optional). */
+int dkv_rebudget(dkv_ctx* ctx, int32_t upto_layer, int32_t* counts_out, void* stream);
+
+/* (4) Algorithm 1's buffer build and truncation for one layer.
+ *     k_src, v_src != NULL : gather.  kb[b,h,0:c] = k_src[b,h,idx[0:c]], kb[b,h,c:c+ws] = k_src[b,h,P:S],
+ *                            same for v; c = count[b][layer].  k_src, v_src : bf16 [Bt, Hkv, S, D].
+ *     k_src == v_src == NULL : shrink kb/vb in place to the current count: rows whose rank is below
+ *                            count[b][layer] stay, in position order, followed by the ws window rows.
+ *     kb, vb  : bf16 [Bt, Hkv, Bl' + ws, D] fixed stride; rows past the valid length are unspecified.
+ *     len_out : int32 [Bt, Hkv] valid rows including the window (optional).
+ *     The context's kept indices and ranks are compacted with the rows. */
+int dkv_compact(dkv_ctx* ctx, int32_t layer, const void* k_src, const void* v_src, void* kb, void* vb,
+                int32_t* len_out, void* stream);
+
+/* Shrink (as above) the buffers of all layers [0, upto_layer) in one launch.
+ * kb, vb : HOST arrays of upto_layer device pointers. */
+int dkv_compact_all(dkv_ctx* ctx, int32_t upto_layer, void* const* kb, void* const* vb, void* stream);
+
+/* Algorithm 1's loop over all L layers: score, select, gather each layer; after every m-th layer (and
+ * after the last one if L % m != 0) rebudget and shrink all preceding layers.  Resets the context first.
+ * q_win, k, v, kb, vb : HOST arrays of L device pointers (layouts as above). */
+int dkv_run_prefill_pass(dkv_ctx* ctx, const void* const* q_win, const void* const* k, const void* const* v,
+                         void* const* kb, void* const* vb, void* stream);
+
+/* The same pass with all tensors in HOST memory (pinned memory recommended): each layer's q, k, v
+ * are copied to device staging buffers owned by the context, processed, and after the last update
+ * every layer's kb/vb (full fixed-stride buffers) and the counts are copied back.  Synchronises.
+ * q_win, k, v, kb, vb : host arrays of L HOST pointers; counts_out : host int32 [Bt, L]. */
+int dkv_run_prefill_pass_host(dkv_ctx* ctx, const void* const* q_win, const void* const* k,
+                              const void* const* v, void* const* kb, void* const* vb, int32_t* counts_out);
+
+/* Copy the current counts to host int32 [Bt, L] (synchronises `stream`). */
+int dkv_get_counts(dkv_ctx* ctx, int32_t* host_counts, void* stream);
+/* Device-side views for inspection, owned by the context: the history scores of a layer
+ * (fp32 [Bt,Hkv,P]) and its current kept positions / ranks (int32 [Bt,Hkv,Bl'], the first
+ * held[b][layer] entries of each head valid).  Any of the out pointers may be NULL. */
+int dkv_layer_views(dkv_ctx* ctx, int32_t layer, const float** scores, const int32_t** idx, const int32_t** rank);
+/* Device-side views of the last update's intermediate integers, int32 [Bt, L] each:
+ * cnt (Eq. 4 hits per layer), Z (Eq. 5), Zp (Eq. 6), and held (rows each layer's buffers hold now). */
+int dkv_budget_views(dkv_ctx* ctx, const int32_t** cnt, const int32_t** z, const int32_t** zp, const int32_t** held);
+/* Copy the status words to host int32 [8] (synchronises the device):
+ * [0] first device-side error (0 = none), [1] kernels launched since dkv_create (host counter). */
+int dkv_last_status(dkv_ctx* ctx, int32_t* host_status);
+/* CUDA error code of the last DKV_ERR_CUDA on this context (0 = none). */
+int dkv_last_cuda_error(dkv_ctx* ctx);
+const char* dkv_strerror(int code);
+/* Library version, 1000*major + minor. */
+int dkv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DKV_H_ */
