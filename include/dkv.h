@@ -137,9 +137,14 @@ int dkv_layer_views(dkv_ctx* ctx, int32_t layer, const float** scores, const int
 /* Device-side views of the last update's intermediate integers, int32 [Bt, L] each:
  * cnt (Eq. 4 hits per layer), Z (Eq. 5), Zp (Eq. 6), and held (rows each layer's buffers hold now). */
 int dkv_budget_views(dkv_ctx* ctx, const int32_t** cnt, const int32_t** z, const int32_t** zp, const int32_t** held);
+/* Convenience for inspecting the views above: copy `bytes` from device memory to host memory and
+ * synchronise `stream`. */
+int dkv_memcpy_to_host(dkv_ctx* ctx, void* host_dst, const void* dev_src, uint64_t bytes, void* stream);
 /* Copy the status words to host int32 [8] (synchronises the device):
  * [0] first device-side error (0 = none), [1] kernels launched since dkv_create (host counter). */
 int dkv_last_status(dkv_ctx* ctx, int32_t* host_status);
+/* Kernels this context has launched since dkv_create (host counter, no synchronisation); -1 if ctx is NULL. */
+int64_t dkv_launch_count(dkv_ctx* ctx);
 /* CUDA error code of the last DKV_ERR_CUDA on this context (0 = none). */
 int dkv_last_cuda_error(dkv_ctx* ctx);
 const char* dkv_strerror(int code);

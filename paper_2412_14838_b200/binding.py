@@ -1,0 +1,229 @@
+"""ctypes view of libdkv.so: the same entry points as include/dkv.h, argument marshalling only.
+
+Every step of the path runs inside the CUDA library; this module converts torch tensors (or raw
+integer addresses) to pointers, passes the current CUDA stream, and raises ``DkvError`` on a
+non-zero return code.  There is no CPU fallback: ``load()`` raises when the library is missing.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libdkv.so")
+
+EXPORTS = [
+    "dkv_create", "dkv_destroy", "dkv_reset", "dkv_score", "dkv_set_scores", "dkv_select_topk", "dkv_rebudget",
+    "dkv_compact", "dkv_compact_all", "dkv_run_prefill_pass", "dkv_run_prefill_pass_host", "dkv_get_counts",
+    "dkv_layer_views", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status", "dkv_launch_count", "dkv_last_cuda_error",
+    "dkv_strerror", "dkv_version",
+]
+
+DKV_OK, DKV_ERR_INVALID_ARG, DKV_ERR_STATE, DKV_ERR_CUDA = 0, -1, -2, -3
+DKV_ERR_TIMEOUT, DKV_ERR_UNSUPPORTED, DKV_ERR_NOMEM = -4, -5, -6
+
+
+class DkvConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "batch", "seq_len", "window", "pool_kernel",
+        "pool_kind", "avg_budget", "layer_max", "update_interval")] + [("flags", ctypes.c_uint32)]
+
+
+class DkvError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {code} ({strerror(code)})")
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libdkv.so (built by ``paper_2412_14838_b200.build``); fail loudly if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2412_14838_b200.build` "
+                           "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, pp = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_void_p)
+    sig = {
+        "dkv_create": [ctypes.POINTER(DkvConfig), pp],
+        "dkv_destroy": [vp],
+        "dkv_reset": [vp, vp],
+        "dkv_score": [vp, i32, vp, vp, vp, vp],
+        "dkv_set_scores": [vp, i32, vp, vp],
+        "dkv_select_topk": [vp, i32, vp, vp, vp],
+        "dkv_rebudget": [vp, i32, vp, vp],
+        "dkv_compact": [vp, i32, vp, vp, vp, vp, vp, vp],
+        "dkv_compact_all": [vp, i32, pp, pp, vp],
+        "dkv_run_prefill_pass": [vp, pp, pp, pp, pp, pp, vp],
+        "dkv_run_prefill_pass_host": [vp, pp, pp, pp, pp, pp, vp],
+        "dkv_get_counts": [vp, vp, vp],
+        "dkv_layer_views": [vp, i32, pp, pp, pp],
+        "dkv_budget_views": [vp, pp, pp, pp, pp],
+        "dkv_memcpy_to_host": [vp, vp, vp, ctypes.c_uint64, vp],
+        "dkv_last_status": [vp, vp],
+        "dkv_last_cuda_error": [vp],
+        "dkv_strerror": [ctypes.c_int],
+        "dkv_version": [],
+        "dkv_launch_count": [vp],
+    }
+    for name, args in sig.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = ctypes.c_int
+    lib.dkv_strerror.restype = ctypes.c_char_p
+    lib.dkv_launch_count.restype = ctypes.c_int64
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().dkv_strerror(code).decode()
+
+
+def _ptr(x) -> Optional[int]:
+    """Address of a torch tensor / numpy array / int; None stays NULL."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):
+        return x.ctypes.data
+    raise TypeError(f"cannot take the address of {type(x)}")
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def _ptr_array(items: Sequence) -> ctypes.Array:
+    arr = (ctypes.c_void_p * len(items))()
+    for i, it in enumerate(items):
+        arr[i] = _ptr(it)
+    return arr
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        raise DkvError(code, what)
+
+
+def make_config(L, Hq, Hkv, D, Bt, S, ws, pool, N, Bl, m, pool_kind=0, flags=0) -> DkvConfig:
+    return DkvConfig(L, Hq, Hkv, D, Bt, S, ws, pool, pool_kind, N, Bl, m, flags)
+
+
+def config_of(w) -> DkvConfig:
+    """DkvConfig of a ``synth.Workload``-like object (fields L,Hq,Hkv,D,Bt,S,ws,pool,N,Bl,m)."""
+    return make_config(w.L, w.Hq, w.Hkv, w.D, w.Bt, w.S, w.ws, w.pool, w.N, w.Bl, w.m)
+
+
+# ---- the entry points, same names as the C ABI ----------------------------------------------------
+def dkv_version() -> int:
+    return load().dkv_version()
+
+
+def dkv_create(cfg: DkvConfig) -> int:
+    h = ctypes.c_void_p()
+    _check(load().dkv_create(ctypes.byref(cfg), ctypes.byref(h)), "dkv_create")
+    return h.value
+
+
+def dkv_destroy(ctx: int) -> None:
+    _check(load().dkv_destroy(ctx), "dkv_destroy")
+
+
+def dkv_reset(ctx: int, stream=None) -> None:
+    _check(load().dkv_reset(ctx, _stream(stream)), "dkv_reset")
+
+
+def dkv_score(ctx: int, layer: int, q_win, k, scores_out=None, stream=None) -> None:
+    _check(load().dkv_score(ctx, layer, _ptr(q_win), _ptr(k), _ptr(scores_out), _stream(stream)), "dkv_score")
+
+
+def dkv_set_scores(ctx: int, layer: int, scores, stream=None) -> None:
+    _check(load().dkv_set_scores(ctx, layer, _ptr(scores), _stream(stream)), "dkv_set_scores")
+
+
+def dkv_select_topk(ctx: int, layer: int, idx_out=None, rank_out=None, stream=None) -> None:
+    _check(load().dkv_select_topk(ctx, layer, _ptr(idx_out), _ptr(rank_out), _stream(stream)), "dkv_select_topk")
+
+
+def dkv_rebudget(ctx: int, upto_layer: int, counts_out=None, stream=None) -> None:
+    _check(load().dkv_rebudget(ctx, upto_layer, _ptr(counts_out), _stream(stream)), "dkv_rebudget")
+
+
+def dkv_compact(ctx: int, layer: int, k_src, v_src, kb, vb, len_out=None, stream=None) -> None:
+    _check(load().dkv_compact(ctx, layer, _ptr(k_src), _ptr(v_src), _ptr(kb), _ptr(vb), _ptr(len_out),
+                              _stream(stream)), "dkv_compact")
+
+
+def dkv_compact_all(ctx: int, upto_layer: int, kb: Sequence, vb: Sequence, stream=None) -> None:
+    _check(load().dkv_compact_all(ctx, upto_layer, _ptr_array(kb), _ptr_array(vb), _stream(stream)),
+           "dkv_compact_all")
+
+
+def dkv_run_prefill_pass(ctx: int, q_win: Sequence, k: Sequence, v: Sequence, kb: Sequence, vb: Sequence,
+                         stream=None) -> None:
+    _check(load().dkv_run_prefill_pass(ctx, _ptr_array(q_win), _ptr_array(k), _ptr_array(v), _ptr_array(kb),
+                                       _ptr_array(vb), _stream(stream)), "dkv_run_prefill_pass")
+
+
+def dkv_run_prefill_pass_host(ctx: int, q_win: Sequence, k: Sequence, v: Sequence, kb: Sequence, vb: Sequence,
+                              counts_out=None) -> None:
+    _check(load().dkv_run_prefill_pass_host(ctx, _ptr_array(q_win), _ptr_array(k), _ptr_array(v), _ptr_array(kb),
+                                            _ptr_array(vb), _ptr(counts_out)), "dkv_run_prefill_pass_host")
+
+
+def dkv_get_counts(ctx: int, host_counts, stream=None) -> None:
+    _check(load().dkv_get_counts(ctx, _ptr(host_counts), _stream(stream)), "dkv_get_counts")
+
+
+def dkv_layer_views(ctx: int, layer: int):
+    """Device addresses (scores, idx, rank) of one layer's state inside the context."""
+    a, b, c = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_void_p()
+    _check(load().dkv_layer_views(ctx, layer, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)), "dkv_layer_views")
+    return a.value, b.value, c.value
+
+
+def dkv_budget_views(ctx: int):
+    """Device addresses (cnt, Z, Z', held), int32 [Bt, L] each."""
+    v = [ctypes.c_void_p() for _ in range(4)]
+    _check(load().dkv_budget_views(ctx, *[ctypes.byref(x) for x in v]), "dkv_budget_views")
+    return tuple(x.value for x in v)
+
+
+def dkv_memcpy_to_host(ctx: int, host_dst, dev_src: int, nbytes: int, stream=None) -> None:
+    _check(load().dkv_memcpy_to_host(ctx, _ptr(host_dst), dev_src, nbytes, _stream(stream)), "dkv_memcpy_to_host")
+
+
+def read_device_i32(ctx: int, dev_src: int, shape):
+    """numpy int32 copy of a device view returned by dkv_layer_views / dkv_budget_views."""
+    import numpy as np
+    out = np.empty(shape, dtype=np.int32)
+    dkv_memcpy_to_host(ctx, out, dev_src, out.nbytes)
+    return out
+
+
+def dkv_last_status(ctx: int):
+    buf = (ctypes.c_int32 * 8)()
+    code = load().dkv_last_status(ctx, buf)
+    return code, list(buf)
+
+
+def dkv_launch_count(ctx: int) -> int:
+    return int(load().dkv_launch_count(ctx))
+
+
+def dkv_last_cuda_error(ctx: int) -> int:
+    return load().dkv_last_cuda_error(ctx)

@@ -1,0 +1,518 @@
+// libdkv: context, argument checking and the C ABI declared in include/dkv.h.
+// The method's steps (Algorithm 1 of arXiv 2412.14838) live in the kernel headers included here.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <new>
+
+#include "../../include/dkv.h"
+#include "common.cuh"
+#include "compact.cuh"
+#include "rebudget.cuh"
+#include "score_simt.cuh"
+#include "select.cuh"
+
+using namespace dkv;
+
+struct dkv_ctx {
+  dkv_config cfg;
+  Shape s;
+  int device;
+  // device state
+  float* d_scores;      // [L][Bt][Hkv][P]  pooled scores, the history A^b
+  float* d_raw;         // [Bt][Hkv][P]     un-pooled scores of the layer being scored
+  int* d_idx;           // [L][Bt][Hkv][Blc] kept positions, ascending
+  int* d_rank;          // [L][Bt][Hkv][Blc] their ranks
+  int* d_count;         // [Bt][L] budget of each layer
+  int* d_held;          // [Bt][L] rows the layer's buffers hold
+  int* d_dbg;           // 3 x [Bt][L] : cnt, Z, Z' of the last update
+  float2* d_stats;      // [Bt*Hkv][n_split][m_stride] partial softmax statistics
+  RbState* d_rb_state;  // [Bt]
+  unsigned int* d_rb_hist;   // [3][Bt][2048]
+  unsigned int* d_cnt_gt;    // [Bt][L]
+  unsigned int* d_cnt_eq;    // [Bt][L]
+  int* d_status;        // [8]
+  int n_split, keys_per_split, m_stride, emit_ctas, keys_per_emit;
+  int sort_n;
+  // host state
+  uint8_t scored[DKV_MAX_LAYERS], selected[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
+  long long launches;
+  int last_cuda;
+  // staging for the host-buffer pass (allocated on first use)
+  bool staged;
+  void *st_q[2], *st_k[2], *st_v[2];
+  void *st_kb[DKV_MAX_LAYERS], *st_vb[DKV_MAX_LAYERS];
+  cudaStream_t st_copy, st_comp;
+  cudaEvent_t ev_copied[2], ev_consumed[2];
+};
+
+namespace {
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int cuda_fail(dkv_ctx* c, cudaError_t e) {
+  if (c) c->last_cuda = (int)e;
+  return e == cudaErrorMemoryAllocation ? DKV_ERR_NOMEM : DKV_ERR_CUDA;
+}
+#define DKV_CUDA(ctx, call)                                   \
+  do {                                                        \
+    cudaError_t e__ = (call);                                 \
+    if (e__ != cudaSuccess) return cuda_fail((ctx), e__);     \
+  } while (0)
+#define DKV_LAUNCHED(ctx)                                     \
+  do {                                                        \
+    (ctx)->launches++;                                        \
+    cudaError_t e__ = cudaPeekAtLastError();                  \
+    if (e__ != cudaSuccess) return cuda_fail((ctx), e__);     \
+  } while (0)
+
+size_t layer_scores(const Shape& s) { return (size_t)s.Bt * s.Hkv * s.P; }
+size_t layer_idx(const Shape& s) { return (size_t)s.Bt * s.Hkv * s.Blc; }
+size_t layer_kv_bytes(const Shape& s) { return (size_t)s.Bt * s.Hkv * s.S * s.D * 2; }
+size_t layer_q_bytes(const Shape& s) { return (size_t)s.Bt * s.Hq * s.ws * s.D * 2; }
+size_t layer_buf_bytes(const Shape& s) { return (size_t)s.Bt * s.Hkv * s.rows * s.D * 2; }
+
+int validate(const dkv_config* c) {
+  if (!c) return DKV_ERR_INVALID_ARG;
+  if (c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->batch < 1) return DKV_ERR_INVALID_ARG;
+  if (c->n_q_heads % c->n_kv_heads != 0) return DKV_ERR_INVALID_ARG;
+  if (c->window < 1 || c->seq_len <= c->window) return DKV_ERR_INVALID_ARG;
+  if (c->pool_kernel < 1 || c->pool_kernel % 2 == 0) return DKV_ERR_INVALID_ARG;
+  if (c->avg_budget < 1 || c->layer_max < c->avg_budget || c->update_interval < 1) return DKV_ERR_INVALID_ARG;
+  if (c->flags != 0) return DKV_ERR_INVALID_ARG;
+  if (c->pool_kind != 0) return DKV_ERR_UNSUPPORTED;
+  if (c->n_layers > DKV_MAX_LAYERS || c->layer_max > DKV_MAX_LAYER_BUDGET) return DKV_ERR_UNSUPPORTED;
+  if (c->head_dim != 64 && c->head_dim != 128) return DKV_ERR_UNSUPPORTED;
+  if ((long long)c->window * (c->n_q_heads / c->n_kv_heads) > DKV_MAX_WINDOW_ROWS) return DKV_ERR_UNSUPPORTED;
+  if ((long long)c->n_layers * c->batch * c->n_kv_heads * (long long)c->seq_len >= (1ll << 31)) return DKV_ERR_UNSUPPORTED;
+  return DKV_OK;
+}
+
+int check_layer(const dkv_ctx* c, int layer) {
+  if (!c) return DKV_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= c->s.L) return DKV_ERR_INVALID_ARG;
+  return DKV_OK;
+}
+
+// ---- step (1): scores of one layer -------------------------------------------------------------
+int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
+  const Shape& s = c->s;
+  const uint16_t* qp = static_cast<const uint16_t*>(q);
+  const uint16_t* kp = static_cast<const uint16_t*>(k);
+  const dim3 g1(c->n_split, s.Bt * s.Hkv), g2(c->emit_ctas, s.Bt * s.Hkv);
+  const int threads = c->m_stride;
+  if (s.D == 128) {
+    score_stats_simt<128><<<g1, threads, 0, st>>>(qp, kp, c->d_stats, s, c->keys_per_split, c->n_split, c->m_stride);
+    DKV_LAUNCHED(c);
+    score_emit_simt<128><<<g2, threads, 0, st>>>(qp, kp, c->d_stats, c->d_raw, s, c->keys_per_emit, c->n_split, c->m_stride);
+    DKV_LAUNCHED(c);
+  } else {
+    score_stats_simt<64><<<g1, threads, 0, st>>>(qp, kp, c->d_stats, s, c->keys_per_split, c->n_split, c->m_stride);
+    DKV_LAUNCHED(c);
+    score_emit_simt<64><<<g2, threads, 0, st>>>(qp, kp, c->d_stats, c->d_raw, s, c->keys_per_emit, c->n_split, c->m_stride);
+    DKV_LAUNCHED(c);
+  }
+  const size_t total = layer_scores(s);
+  maxpool_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(c->d_raw, c->d_scores + (size_t)layer * total, scores_out,
+                                                                  s.P, s.pool / 2, total);
+  DKV_LAUNCHED(c);
+  c->scored[layer] = 1;
+  c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
+  return DKV_OK;
+}
+
+// ---- step (2): per-head top-Bl' ----------------------------------------------------------------
+int do_select(dkv_ctx* c, int layer, int* idx_out, int* rank_out, cudaStream_t st) {
+  const Shape& s = c->s;
+  select_topk_kernel<<<s.Bt * s.Hkv, kSelThreads, (size_t)c->sort_n * 8, st>>>(
+      c->d_scores + (size_t)layer * layer_scores(s), c->d_idx + (size_t)layer * layer_idx(s),
+      c->d_rank + (size_t)layer * layer_idx(s), idx_out, rank_out, s.P, s.Blc, c->sort_n, c->d_count, s.Hkv, s.L, layer);
+  DKV_LAUNCHED(c);
+  c->selected[layer] = 1;
+  c->gathered[layer] = c->stale[layer] = 0;
+  return DKV_OK;
+}
+
+// ---- step (3): Update_Buffer_Length ------------------------------------------------------------
+int do_rebudget(dkv_ctx* c, int l, int* counts_out, cudaStream_t st) {
+  const Shape& s = c->s;
+  const size_t per_layer = (size_t)s.Hkv * s.P;
+  long long k = (long long)s.N * s.Hkv * l;
+  const long long pop = (long long)l * (long long)per_layer;
+  if (k > pop) k = pop;
+  const int init_n = 3 * s.Bt * kRbBins > s.Bt * s.L ? 3 * s.Bt * kRbBins : s.Bt * s.L;
+  rb_init_kernel<<<(init_n + 255) / 256, 256, 0, st>>>(c->d_rb_state, c->d_rb_hist, c->d_cnt_gt, c->d_cnt_eq, s.Bt, s.L,
+                                                      (unsigned int)k);
+  DKV_LAUNCHED(c);
+  int bpl = (int)((per_layer + (size_t)kRbThreads * 8 - 1) / ((size_t)kRbThreads * 8));
+  if (bpl > 64) bpl = 64;
+  if (bpl < 1) bpl = 1;
+  const dim3 grid(bpl, l, s.Bt);
+  for (int pass = 0; pass < 3; ++pass) {
+    rb_hist_kernel<<<grid, kRbThreads, 0, st>>>(c->d_scores, c->d_rb_state, c->d_rb_hist, pass, s.Bt, per_layer);
+    DKV_LAUNCHED(c);
+    rb_scan_kernel<<<s.Bt, 1024, 0, st>>>(c->d_rb_state, c->d_rb_hist, pass, s.Bt);
+    DKV_LAUNCHED(c);
+  }
+  rb_count_kernel<<<grid, kRbThreads, 0, st>>>(c->d_scores, c->d_rb_state, c->d_cnt_gt, c->d_cnt_eq, s.Bt, s.L, per_layer);
+  DKV_LAUNCHED(c);
+  const size_t bl = (size_t)s.Bt * s.L;
+  rb_budget_kernel<<<(s.Bt + 31) / 32, 32, 0, st>>>(c->d_cnt_gt, c->d_cnt_eq, c->d_count, c->d_dbg, c->d_dbg + bl,
+                                                   c->d_dbg + 2 * bl, counts_out, s.Bt, s.L, l, k, s.Bl, s.N);
+  DKV_LAUNCHED(c);
+  for (int i = 0; i < l; ++i) if (!c->gathered[i]) c->stale[i] = 1;
+  return DKV_OK;
+}
+
+// ---- step (4): gather / shrink ------------------------------------------------------------------
+int do_shrink(dkv_ctx* c, int layer0, int n, void* const* kb, void* const* vb, cudaStream_t st) {
+  const Shape& s = c->s;
+  LayerPtrs ptrs;
+  for (int i = 0; i < n; ++i) { ptrs.kb[layer0 + i] = kb[i]; ptrs.vb[layer0 + i] = vb[i]; }
+  shrink_kernel<<<dim3(s.Bt * s.Hkv, n), kShrinkThreads, (size_t)s.Blc * 4, st>>>(
+      ptrs, layer0, c->d_idx, c->d_rank, c->d_count, c->d_held, s.Bt, s.Hkv, s.L, s.ws, s.Blc, s.rows, s.D * 2 / 16,
+      layer_idx(s));
+  DKV_LAUNCHED(c);
+  commit_held_kernel<<<(s.Bt * n + 127) / 128, 128, 0, st>>>(c->d_held, c->d_count, s.Bt, s.L, layer0, n);
+  DKV_LAUNCHED(c);
+  return DKV_OK;
+}
+
+int do_gather(dkv_ctx* c, int layer, const void* k_src, const void* v_src, void* kb, void* vb, cudaStream_t st) {
+  const Shape& s = c->s;
+  const int vec = s.D * 2 / 16, rpb = 256 / vec;
+  const dim3 grid((s.rows + rpb - 1) / rpb, s.Bt * s.Hkv, 2);
+  gather_rows_kernel<<<grid, 256, 0, st>>>(static_cast<const uint4*>(k_src), static_cast<const uint4*>(v_src),
+                                           static_cast<uint4*>(kb), static_cast<uint4*>(vb),
+                                           c->d_idx + (size_t)layer * layer_idx(s), s.Blc, s.S, s.P, s.ws, s.rows, vec,
+                                           c->d_held, s.Hkv, s.L, layer);
+  DKV_LAUNCHED(c);
+  c->gathered[layer] = 1;
+  if (c->stale[layer]) {           // an update ran between select and gather: apply it now
+    c->stale[layer] = 0;
+    return do_shrink(c, layer, 1, &kb, &vb, st);
+  }
+  return DKV_OK;
+}
+
+int do_reset(dkv_ctx* c, cudaStream_t st) {
+  const Shape& s = c->s;
+  DKV_CUDA(c, cudaMemsetAsync(c->d_count, 0, sizeof(int) * s.Bt * s.L, st));
+  DKV_CUDA(c, cudaMemsetAsync(c->d_held, 0, sizeof(int) * s.Bt * s.L, st));
+  DKV_CUDA(c, cudaMemsetAsync(c->d_dbg, 0, sizeof(int) * 3 * s.Bt * s.L, st));
+  memset(c->scored, 0, sizeof c->scored);
+  memset(c->selected, 0, sizeof c->selected);
+  memset(c->gathered, 0, sizeof c->gathered);
+  memset(c->stale, 0, sizeof c->stale);
+  return DKV_OK;
+}
+
+int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* const* v, void* const* kb,
+            void* const* vb, cudaStream_t st) {
+  const Shape& s = c->s;
+  int rc = do_reset(c, st);
+  if (rc) return rc;
+  for (int l = 0; l < s.L; ++l) {
+    if ((rc = do_score(c, l, q[l], k[l], nullptr, st))) return rc;
+    if ((rc = do_select(c, l, nullptr, nullptr, st))) return rc;
+    if ((rc = do_gather(c, l, k[l], v[l], kb[l], vb[l], st))) return rc;
+    const bool update = ((l + 1) % s.m == 0) || (l + 1 == s.L && s.L % s.m != 0);
+    if (update) {
+      if ((rc = do_rebudget(c, l + 1, nullptr, st))) return rc;
+      if ((rc = do_shrink(c, 0, l + 1, kb, vb, st))) return rc;
+    }
+  }
+  return DKV_OK;
+}
+
+void free_all(dkv_ctx* c) {
+  cudaFree(c->d_scores); cudaFree(c->d_raw); cudaFree(c->d_idx); cudaFree(c->d_rank); cudaFree(c->d_count);
+  cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_stats); cudaFree(c->d_rb_state); cudaFree(c->d_rb_hist);
+  cudaFree(c->d_cnt_gt); cudaFree(c->d_cnt_eq); cudaFree(c->d_status);
+  if (c->staged) {
+    for (int i = 0; i < 2; ++i) {
+      cudaFree(c->st_q[i]); cudaFree(c->st_k[i]); cudaFree(c->st_v[i]);
+      cudaEventDestroy(c->ev_copied[i]); cudaEventDestroy(c->ev_consumed[i]);
+    }
+    for (int l = 0; l < c->s.L; ++l) { cudaFree(c->st_kb[l]); cudaFree(c->st_vb[l]); }
+    cudaStreamDestroy(c->st_copy); cudaStreamDestroy(c->st_comp);
+  }
+}
+
+int ensure_staging(dkv_ctx* c) {
+  if (c->staged) return DKV_OK;
+  const Shape& s = c->s;
+  for (int i = 0; i < 2; ++i) {
+    DKV_CUDA(c, cudaMalloc(&c->st_q[i], layer_q_bytes(s)));
+    DKV_CUDA(c, cudaMalloc(&c->st_k[i], layer_kv_bytes(s)));
+    DKV_CUDA(c, cudaMalloc(&c->st_v[i], layer_kv_bytes(s)));
+    DKV_CUDA(c, cudaEventCreateWithFlags(&c->ev_copied[i], cudaEventDisableTiming));
+    DKV_CUDA(c, cudaEventCreateWithFlags(&c->ev_consumed[i], cudaEventDisableTiming));
+  }
+  for (int l = 0; l < s.L; ++l) {
+    DKV_CUDA(c, cudaMalloc(&c->st_kb[l], layer_buf_bytes(s)));
+    DKV_CUDA(c, cudaMalloc(&c->st_vb[l], layer_buf_bytes(s)));
+  }
+  DKV_CUDA(c, cudaStreamCreateWithFlags(&c->st_copy, cudaStreamNonBlocking));
+  DKV_CUDA(c, cudaStreamCreateWithFlags(&c->st_comp, cudaStreamNonBlocking));
+  c->staged = true;
+  return DKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dkv_version(void) { return 1000; }
+
+const char* dkv_strerror(int code) {
+  switch (code) {
+    case DKV_OK: return "ok";
+    case DKV_ERR_INVALID_ARG: return "invalid argument";
+    case DKV_ERR_STATE: return "call out of order for this layer";
+    case DKV_ERR_CUDA: return "CUDA runtime error";
+    case DKV_ERR_TIMEOUT: return "device-side wait timed out";
+    case DKV_ERR_UNSUPPORTED: return "shape not supported";
+    case DKV_ERR_NOMEM: return "out of memory";
+    default: return "unknown error";
+  }
+}
+
+int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
+  if (!out) return DKV_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = validate(cfg);
+  if (rc) return rc;
+  dkv_ctx* c = new (std::nothrow) dkv_ctx;
+  if (!c) return DKV_ERR_NOMEM;
+  memset(c, 0, sizeof *c);
+  c->cfg = *cfg;
+  Shape& s = c->s;
+  s.L = cfg->n_layers; s.Hq = cfg->n_q_heads; s.Hkv = cfg->n_kv_heads; s.D = cfg->head_dim; s.Bt = cfg->batch;
+  s.S = cfg->seq_len; s.ws = cfg->window; s.pool = cfg->pool_kernel; s.N = cfg->avg_budget; s.Bl = cfg->layer_max;
+  s.m = cfg->update_interval;
+  s.G = s.Hq / s.Hkv; s.P = s.S - s.ws; s.M = s.ws * s.G; s.Blc = s.Bl < s.P ? s.Bl : s.P; s.rows = s.Blc + s.ws;
+  c->m_stride = (s.M + 31) / 32 * 32;
+  const int heads = s.Bt * s.Hkv;
+  int split = (4 * 148 + heads - 1) / heads;
+  if (split > 64) split = 64;
+  int kps = ((s.S + split - 1) / split + kSimtTileKeys - 1) / kSimtTileKeys * kSimtTileKeys;
+  c->keys_per_split = kps;
+  c->n_split = (s.S + kps - 1) / kps;
+  int kpe = ((s.P + split - 1) / split + kSimtTileKeys - 1) / kSimtTileKeys * kSimtTileKeys;
+  c->keys_per_emit = kpe;
+  c->emit_ctas = (s.P + kpe - 1) / kpe;
+  c->sort_n = 2;
+  while (c->sort_n < s.Blc) c->sort_n <<= 1;
+
+  cudaError_t e = cudaGetDevice(&c->device);
+  const size_t bl = (size_t)s.Bt * s.L;
+#define TRY(call) if (e == cudaSuccess) e = (call)
+  TRY(cudaMalloc(&c->d_scores, sizeof(float) * s.L * layer_scores(s)));
+  TRY(cudaMalloc(&c->d_raw, sizeof(float) * layer_scores(s)));
+  TRY(cudaMalloc(&c->d_idx, sizeof(int) * s.L * layer_idx(s)));
+  TRY(cudaMalloc(&c->d_rank, sizeof(int) * s.L * layer_idx(s)));
+  TRY(cudaMalloc(&c->d_count, sizeof(int) * bl));
+  TRY(cudaMalloc(&c->d_held, sizeof(int) * bl));
+  TRY(cudaMalloc(&c->d_dbg, sizeof(int) * 3 * bl));
+  TRY(cudaMalloc(&c->d_stats, sizeof(float2) * heads * c->n_split * c->m_stride));
+  TRY(cudaMalloc(&c->d_rb_state, sizeof(RbState) * s.Bt));
+  TRY(cudaMalloc(&c->d_rb_hist, sizeof(unsigned int) * 3 * s.Bt * kRbBins));
+  TRY(cudaMalloc(&c->d_cnt_gt, sizeof(unsigned int) * bl));
+  TRY(cudaMalloc(&c->d_cnt_eq, sizeof(unsigned int) * bl));
+  TRY(cudaMalloc(&c->d_status, sizeof(int) * 8));
+  TRY(cudaMemset(c->d_status, 0, sizeof(int) * 8));
+  TRY(cudaMemset(c->d_count, 0, sizeof(int) * bl));
+  TRY(cudaMemset(c->d_held, 0, sizeof(int) * bl));
+  TRY(cudaMemset(c->d_dbg, 0, sizeof(int) * 3 * bl));
+  TRY(cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, c->sort_n * 8));
+  TRY(cudaFuncSetAttribute(shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, s.Blc * 4));
+#undef TRY
+  if (e != cudaSuccess) {
+    rc = e == cudaErrorMemoryAllocation ? DKV_ERR_NOMEM : DKV_ERR_CUDA;
+    cudaGetLastError();
+    free_all(c);
+    delete c;
+    return rc;
+  }
+  *out = c;
+  return DKV_OK;
+}
+
+int dkv_destroy(dkv_ctx* c) {
+  if (!c) return DKV_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  free_all(c);
+  delete c;
+  return DKV_OK;
+}
+
+int dkv_reset(dkv_ctx* c, void* stream) {
+  if (!c) return DKV_ERR_INVALID_ARG;
+  return do_reset(c, as_stream(stream));
+}
+
+int dkv_score(dkv_ctx* c, int32_t layer, const void* q_win, const void* k, float* scores_out, void* stream) {
+  int rc = check_layer(c, layer);
+  if (rc) return rc;
+  if (!q_win || !k || !aligned16(q_win) || !aligned16(k) || !aligned16(scores_out)) return DKV_ERR_INVALID_ARG;
+  return do_score(c, layer, q_win, k, scores_out, as_stream(stream));
+}
+
+int dkv_set_scores(dkv_ctx* c, int32_t layer, const float* scores, void* stream) {
+  int rc = check_layer(c, layer);
+  if (rc) return rc;
+  if (!scores) return DKV_ERR_INVALID_ARG;
+  const size_t n = layer_scores(c->s);
+  DKV_CUDA(c, cudaMemcpyAsync(c->d_scores + (size_t)layer * n, scores, n * sizeof(float), cudaMemcpyDeviceToDevice,
+                              as_stream(stream)));
+  c->scored[layer] = 1;
+  c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
+  return DKV_OK;
+}
+
+int dkv_select_topk(dkv_ctx* c, int32_t layer, int32_t* idx_out, int32_t* rank_out, void* stream) {
+  int rc = check_layer(c, layer);
+  if (rc) return rc;
+  if (!c->scored[layer]) return DKV_ERR_STATE;
+  return do_select(c, layer, idx_out, rank_out, as_stream(stream));
+}
+
+int dkv_rebudget(dkv_ctx* c, int32_t upto_layer, int32_t* counts_out, void* stream) {
+  if (!c || upto_layer < 1 || upto_layer > c->s.L) return DKV_ERR_INVALID_ARG;
+  for (int i = 0; i < upto_layer; ++i) if (!c->scored[i] || !c->selected[i]) return DKV_ERR_STATE;
+  return do_rebudget(c, upto_layer, counts_out, as_stream(stream));
+}
+
+int dkv_compact(dkv_ctx* c, int32_t layer, const void* k_src, const void* v_src, void* kb, void* vb, int32_t* len_out,
+                void* stream) {
+  int rc = check_layer(c, layer);
+  if (rc) return rc;
+  if (!kb || !vb || !aligned16(kb) || !aligned16(vb)) return DKV_ERR_INVALID_ARG;
+  if ((k_src == nullptr) != (v_src == nullptr)) return DKV_ERR_INVALID_ARG;
+  if (!aligned16(k_src) || !aligned16(v_src)) return DKV_ERR_INVALID_ARG;
+  cudaStream_t st = as_stream(stream);
+  if (k_src) {
+    if (!c->selected[layer]) return DKV_ERR_STATE;
+    rc = do_gather(c, layer, k_src, v_src, kb, vb, st);
+  } else {
+    if (!c->gathered[layer]) return DKV_ERR_STATE;
+    rc = do_shrink(c, layer, 1, &kb, &vb, st);
+  }
+  if (rc) return rc;
+  if (len_out) {
+    const Shape& s = c->s;
+    write_len_kernel<<<(s.Bt * s.Hkv + 127) / 128, 128, 0, st>>>(len_out, c->d_held, s.Bt, s.Hkv, s.L, layer, s.ws);
+    DKV_LAUNCHED(c);
+  }
+  return DKV_OK;
+}
+
+int dkv_compact_all(dkv_ctx* c, int32_t upto_layer, void* const* kb, void* const* vb, void* stream) {
+  if (!c || !kb || !vb || upto_layer < 1 || upto_layer > c->s.L) return DKV_ERR_INVALID_ARG;
+  for (int i = 0; i < upto_layer; ++i) {
+    if (!kb[i] || !vb[i] || !aligned16(kb[i]) || !aligned16(vb[i])) return DKV_ERR_INVALID_ARG;
+    if (!c->gathered[i]) return DKV_ERR_STATE;
+  }
+  return do_shrink(c, 0, upto_layer, kb, vb, as_stream(stream));
+}
+
+int dkv_run_prefill_pass(dkv_ctx* c, const void* const* q_win, const void* const* k, const void* const* v,
+                         void* const* kb, void* const* vb, void* stream) {
+  if (!c || !q_win || !k || !v || !kb || !vb) return DKV_ERR_INVALID_ARG;
+  for (int l = 0; l < c->s.L; ++l) {
+    if (!q_win[l] || !k[l] || !v[l] || !kb[l] || !vb[l]) return DKV_ERR_INVALID_ARG;
+    if (!aligned16(q_win[l]) || !aligned16(k[l]) || !aligned16(v[l]) || !aligned16(kb[l]) || !aligned16(vb[l]))
+      return DKV_ERR_INVALID_ARG;
+  }
+  return do_pass(c, q_win, k, v, kb, vb, as_stream(stream));
+}
+
+int dkv_run_prefill_pass_host(dkv_ctx* c, const void* const* q_win, const void* const* k, const void* const* v,
+                              void* const* kb, void* const* vb, int32_t* counts_out) {
+  if (!c || !q_win || !k || !v || !kb || !vb) return DKV_ERR_INVALID_ARG;
+  const Shape& s = c->s;
+  for (int l = 0; l < s.L; ++l)
+    if (!q_win[l] || !k[l] || !v[l] || !kb[l] || !vb[l]) return DKV_ERR_INVALID_ARG;
+  int rc = ensure_staging(c);
+  if (rc) return rc;
+  cudaStream_t cp = c->st_copy, st = c->st_comp;
+  if ((rc = do_reset(c, st))) return rc;
+  for (int l = 0; l < s.L; ++l) {
+    const int slot = l & 1;
+    if (l >= 2) DKV_CUDA(c, cudaStreamWaitEvent(cp, c->ev_consumed[slot], 0));
+    DKV_CUDA(c, cudaMemcpyAsync(c->st_q[slot], q_win[l], layer_q_bytes(s), cudaMemcpyHostToDevice, cp));
+    DKV_CUDA(c, cudaMemcpyAsync(c->st_k[slot], k[l], layer_kv_bytes(s), cudaMemcpyHostToDevice, cp));
+    DKV_CUDA(c, cudaMemcpyAsync(c->st_v[slot], v[l], layer_kv_bytes(s), cudaMemcpyHostToDevice, cp));
+    DKV_CUDA(c, cudaEventRecord(c->ev_copied[slot], cp));
+    DKV_CUDA(c, cudaStreamWaitEvent(st, c->ev_copied[slot], 0));
+    if ((rc = do_score(c, l, c->st_q[slot], c->st_k[slot], nullptr, st))) return rc;
+    if ((rc = do_select(c, l, nullptr, nullptr, st))) return rc;
+    if ((rc = do_gather(c, l, c->st_k[slot], c->st_v[slot], c->st_kb[l], c->st_vb[l], st))) return rc;
+    DKV_CUDA(c, cudaEventRecord(c->ev_consumed[slot], st));
+    const bool update = ((l + 1) % s.m == 0) || (l + 1 == s.L && s.L % s.m != 0);
+    if (update) {
+      if ((rc = do_rebudget(c, l + 1, nullptr, st))) return rc;
+      if ((rc = do_shrink(c, 0, l + 1, c->st_kb, c->st_vb, st))) return rc;
+    }
+  }
+  for (int l = 0; l < s.L; ++l) {
+    DKV_CUDA(c, cudaMemcpyAsync(kb[l], c->st_kb[l], layer_buf_bytes(s), cudaMemcpyDeviceToHost, st));
+    DKV_CUDA(c, cudaMemcpyAsync(vb[l], c->st_vb[l], layer_buf_bytes(s), cudaMemcpyDeviceToHost, st));
+  }
+  if (counts_out)
+    DKV_CUDA(c, cudaMemcpyAsync(counts_out, c->d_count, sizeof(int) * s.Bt * s.L, cudaMemcpyDeviceToHost, st));
+  DKV_CUDA(c, cudaStreamSynchronize(cp));
+  DKV_CUDA(c, cudaStreamSynchronize(st));
+  return DKV_OK;
+}
+
+int dkv_get_counts(dkv_ctx* c, int32_t* host_counts, void* stream) {
+  if (!c || !host_counts) return DKV_ERR_INVALID_ARG;
+  DKV_CUDA(c, cudaMemcpyAsync(host_counts, c->d_count, sizeof(int) * c->s.Bt * c->s.L, cudaMemcpyDeviceToHost,
+                              as_stream(stream)));
+  DKV_CUDA(c, cudaStreamSynchronize(as_stream(stream)));
+  return DKV_OK;
+}
+
+int dkv_layer_views(dkv_ctx* c, int32_t layer, const float** scores, const int32_t** idx, const int32_t** rank) {
+  int rc = check_layer(c, layer);
+  if (rc) return rc;
+  if (scores) *scores = c->d_scores + (size_t)layer * layer_scores(c->s);
+  if (idx) *idx = c->d_idx + (size_t)layer * layer_idx(c->s);
+  if (rank) *rank = c->d_rank + (size_t)layer * layer_idx(c->s);
+  return DKV_OK;
+}
+
+int dkv_budget_views(dkv_ctx* c, const int32_t** cnt, const int32_t** z, const int32_t** zp, const int32_t** held) {
+  if (!c) return DKV_ERR_INVALID_ARG;
+  const size_t bl = (size_t)c->s.Bt * c->s.L;
+  if (cnt) *cnt = c->d_dbg;
+  if (z) *z = c->d_dbg + bl;
+  if (zp) *zp = c->d_dbg + 2 * bl;
+  if (held) *held = c->d_held;
+  return DKV_OK;
+}
+
+int dkv_memcpy_to_host(dkv_ctx* c, void* host_dst, const void* dev_src, uint64_t bytes, void* stream) {
+  if (!c || !host_dst || !dev_src) return DKV_ERR_INVALID_ARG;
+  DKV_CUDA(c, cudaMemcpyAsync(host_dst, dev_src, bytes, cudaMemcpyDeviceToHost, as_stream(stream)));
+  DKV_CUDA(c, cudaStreamSynchronize(as_stream(stream)));
+  return DKV_OK;
+}
+
+int dkv_last_status(dkv_ctx* c, int32_t* host_status) {
+  if (!c || !host_status) return DKV_ERR_INVALID_ARG;
+  DKV_CUDA(c, cudaDeviceSynchronize());
+  DKV_CUDA(c, cudaMemcpy(host_status, c->d_status, sizeof(int) * 8, cudaMemcpyDeviceToHost));
+  host_status[1] = (int32_t)(c->launches & 0x7FFFFFFF);
+  return host_status[0] == 0 ? DKV_OK : host_status[0];
+}
+
+int64_t dkv_launch_count(dkv_ctx* c) { return c ? (int64_t)c->launches : -1; }
+
+int dkv_last_cuda_error(dkv_ctx* c) { return c ? c->last_cuda : 0; }
+
+}  // extern "C"

@@ -6,7 +6,7 @@
 
 namespace dkv {
 
-constexpr int kSimtTileKeys = 32;
+constexpr int kSimtTileKeys = 16;
 
 // Partial softmax statistics of one row over one key range, in the base-2 domain:
 // x = running max of t = logit * log2(e)/sqrt(D); y = sum of 2^(t - x).
