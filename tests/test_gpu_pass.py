@@ -1,0 +1,233 @@
+"""End-to-end parity of Algorithm 1's loop (dkv_run_prefill_pass) against the oracle.
+
+Small and medium workloads are compared in full: scores within tolerance; kept sets, counts and
+compacted K/V bytes bit-exact, except where the oracle's own scores are tied at the cut within
+the near-tie gap (such events are counted and printed).  The full-size workloads run in the same
+launch configuration the benchmark times; the oracle checks sampled (layer, head) outputs one by
+one, and properties that hold at any size cover the rest.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dynamickv as O
+from paper_2412_14838_b200 import binding as B
+from paper_2412_14838_b200 import build, synth
+from tests import _util as U
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    B.load()
+
+
+def dev(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda()
+
+
+class GpuPass:
+    """Inputs on the device, one full pass, results back on the host."""
+
+    def __init__(self, w, keep_inputs=True):
+        self.w = w
+        self.q, self.k, self.v = [], [], []
+        self.host = []
+        for l in range(w.L):
+            t = synth.layer_inputs(w, l)
+            self.q.append(dev(t["q"])); self.k.append(dev(t["k"])); self.v.append(dev(t["v"]))
+            self.host.append(t if keep_inputs else None)
+        shape = (w.Bt, w.Hkv, w.Blc + w.ws, w.D)
+        self.kb = [torch.zeros(shape, dtype=torch.int16, device="cuda") for _ in range(w.L)]
+        self.vb = [torch.zeros(shape, dtype=torch.int16, device="cuda") for _ in range(w.L)]
+        self.h = B.dkv_create(B.config_of(w))
+
+    def run(self):
+        B.dkv_run_prefill_pass(self.h, self.q, self.k, self.v, self.kb, self.vb)
+        torch.cuda.synchronize()
+        w = self.w
+        self.counts = np.zeros((w.Bt, w.L), dtype=np.int32)
+        B.dkv_get_counts(self.h, self.counts)
+        self.held = B.read_device_i32(self.h, B.dkv_budget_views(self.h)[3], (w.Bt, w.L))
+        code, status = B.dkv_last_status(self.h)
+        assert code == 0 and status[0] == 0
+        return self
+
+    def scores(self, layer):
+        w = self.w
+        out = np.empty((w.Bt, w.Hkv, w.P), dtype=np.float32)
+        B.dkv_memcpy_to_host(self.h, out, B.dkv_layer_views(self.h, layer)[0], out.nbytes)
+        return out
+
+    def idx_rank(self, layer):
+        w = self.w
+        _, ia, ra = B.dkv_layer_views(self.h, layer)
+        return (B.read_device_i32(self.h, ia, (w.Bt, w.Hkv, w.Blc)), B.read_device_i32(self.h, ra, (w.Bt, w.Hkv, w.Blc)))
+
+    def close(self):
+        B.dkv_destroy(self.h)
+
+
+def check_properties(g: GpuPass):
+    """What must hold at any size, checked from the inputs and the library's own outputs."""
+    w = g.w
+    assert (g.held == g.counts).all(), "buffers were not brought down to the final counts"
+    assert (g.counts >= 0).all() and (g.counts <= w.Blc).all()
+    assert (g.counts.sum(axis=1) <= w.N * w.L).all(), "global budget exceeded"
+    for l in range(w.L):
+        idx, rank = g.idx_rank(l)
+        sc = torch.from_numpy(g.scores(l)).cuda()
+        for b in range(w.Bt):
+            n = int(g.counts[b, l])
+            ii = torch.from_numpy(idx[b, :, :n].astype(np.int64)).cuda()           # [Hkv, n]
+            rr = rank[b, :, :n]
+            assert (np.diff(idx[b, :, :n], axis=1) > 0).all() and (idx[b, :, :n] < w.P).all()
+            assert (np.sort(rr, axis=1) == np.arange(n)[None, :]).all(), "ranks are not 0..n-1"
+            # kept rows and window rows are byte copies of the layer's K/V
+            for src, buf in ((g.k[l], g.kb[l]), (g.v[l], g.vb[l])):
+                want = torch.gather(src[b], 1, ii[:, :, None].expand(-1, -1, w.D))
+                assert torch.equal(buf[b, :, :n], want)
+                assert torch.equal(buf[b, :, n:n + w.ws], src[b, :, w.P:])
+            # every kept score >= every dropped score (per head), order by rank is non-increasing
+            kept = torch.gather(sc[b], 1, ii)
+            mask = torch.ones_like(sc[b], dtype=torch.bool).scatter_(1, ii, False)
+            dropped_max = torch.where(mask, sc[b], torch.full_like(sc[b], -1.0)).max(dim=1).values
+            if n:
+                assert (kept.min(dim=1).values >= dropped_max).all()
+                by_rank = torch.gather(kept, 1, torch.from_numpy(np.argsort(rr, axis=1)).cuda())
+                assert (by_rank[:, 1:] <= by_rank[:, :-1]).all()
+
+
+def compare_full(g: GpuPass, verbose_name=""):
+    """Whole-pass comparison with the oracle, near-ties counted."""
+    w = g.w
+
+    def layer_fn(l):
+        t = g.host[l]
+        return {"q": synth.bf16_bits_to_f64(t["q"]), "k": synth.bf16_bits_to_f64(t["k"]),
+                "k_rows": t["k"], "v_rows": t["v"]}
+
+    ref = O.run_prefill_pass(layer_fn, w.L, ws=w.ws, pool=w.pool, N=w.N, Bl=w.Bl, m=w.m)
+    worst, near = 0.0, 0
+    for l in range(w.L):
+        worst = max(worst, U.assert_scores_close(g.scores(l), ref["score"][l], f"{w.name} layer {l}"))
+    counts_equal = (g.counts == ref["counts"]).all()
+    if not counts_equal:
+        # only a near-tie at some update's global cut may move a count
+        gaps = [U.global_cut_gap([ref["score"][i][b] for i in range(l_done)], w.N * w.Hkv * l_done)
+                for l_done, _ in ref["updates"] for b in range(w.Bt)]
+        assert min(gaps) <= U.NEAR_TIE, f"counts differ ({g.counts} vs {ref['counts']}) without a global near-tie"
+        near += 1
+    for l in range(w.L):
+        idx, _ = g.idx_rank(l)
+        kb = g.kb[l].cpu().numpy().view(np.uint16)
+        vb = g.vb[l].cpu().numpy().view(np.uint16)
+        for b in range(w.Bt):
+            n = int(g.counts[b, l])
+            for h in range(w.Hkv):
+                exact, ev = U.select_matches(ref["score"][l][b, h], idx[b, h, :n], n)
+                near += ev
+                if exact and counts_equal:
+                    assert (kb[b, h, :n + w.ws] == ref["kb"][l][b][h]).all(), f"K bytes differ l={l} h={h}"
+                    assert (vb[b, h, :n + w.ws] == ref["vb"][l][b][h]).all(), f"V bytes differ l={l} h={h}"
+    print(f"[{w.name}] max rel score error {worst:.2e}; near-tie events {near}; counts {g.counts.tolist()}")
+    return near
+
+
+@pytest.mark.parametrize("name", ["tiny", "mistral8k"])
+def test_pass_matches_oracle_in_full(name):
+    w = synth.WORKLOADS[name]
+    g = GpuPass(w).run()
+    try:
+        check_properties(g)
+        near = compare_full(g)
+        assert near <= 8, "implausibly many near-ties"
+    finally:
+        g.close()
+
+
+def test_pass_with_ragged_shape_and_final_partial_block():
+    # L % m != 0 (extra update after the last layer), G = 3, batch 2, odd sizes
+    w = synth.Workload("ragpass", 51, L=5, Hq=6, Hkv=2, D=128, Bt=2, S=1500, ws=8, pool=3, N=24, Bl=60, m=2,
+                       recipe="sink")
+    g = GpuPass(w).run()
+    try:
+        check_properties(g)
+        compare_full(g)
+    finally:
+        g.close()
+
+
+FULL = ["mistral32k", "llama16k_b4", "needle32k"]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_full_size_pass_sampled(name):
+    w = synth.WORKLOADS[name]
+    g = GpuPass(w, keep_inputs=False).run()
+    try:
+        check_properties(g)
+        rng = np.random.default_rng(w.cid)
+        samples = [(int(rng.integers(w.L)), int(rng.integers(w.Bt)), int(rng.integers(w.Hkv))) for _ in range(3)]
+        samples.append((w.L - 1, w.Bt - 1, w.Hkv - 1))
+        near = 0
+        for (l, b, h) in samples:
+            t = synth.layer_inputs(w, l, want_v=False)
+            G = w.G
+            q = synth.bf16_bits_to_f64(t["q"][b:b + 1, h * G:(h + 1) * G])
+            k = synth.bf16_bits_to_f64(t["k"][b:b + 1, h:h + 1])
+            ref = O.window_scores(q, k, w.ws, w.pool)["score"][0, 0]
+            got = g.scores(l)[b, h]
+            U.assert_scores_close(got, ref, f"{name} l={l} b={b} h={h}")
+            n = int(g.counts[b, l])
+            idx, _ = g.idx_rank(l)
+            _, ev = U.select_matches(ref, idx[b, h, :n], n)
+            near += ev
+        print(f"[{name}] sampled heads ok; near-tie events {near}; counts {g.counts.tolist()}")
+        if name == "needle32k":
+            mask = synth.needle_token_mask(w)
+            frac = []
+            for l in range(w.L):
+                idx, _ = g.idx_rank(l)
+                n = int(g.counts[0, l])
+                frac.append(float(np.mean([mask[idx[0, h, :n]].sum() / 128.0 for h in range(w.Hkv)])))
+            print("[needle32k] needle tokens retained per layer:", np.round(frac, 2).tolist())
+            assert max(frac[7:24]) > 0.5, "planted needles are not retained in the layers that carry them"
+    finally:
+        g.close()
+
+
+@pytest.mark.skipif(not os.environ.get("DKV_FULL_ORACLE"), reason="set DKV_FULL_ORACLE=1: minutes of CPU per workload")
+@pytest.mark.parametrize("name", FULL)
+def test_full_size_pass_whole_oracle(name):
+    w = synth.WORKLOADS[name]
+    g = GpuPass(w).run()
+    try:
+        compare_full(g)
+    finally:
+        g.close()
+
+
+def test_host_buffer_pass_matches_device_pass():
+    w = synth.WORKLOADS["tiny"]
+    g = GpuPass(w).run()
+    try:
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+        hq = [pin(t["q"]) for t in g.host]; hk = [pin(t["k"]) for t in g.host]; hv = [pin(t["v"]) for t in g.host]
+        shape = (w.Bt, w.Hkv, w.Blc + w.ws, w.D)
+        okb = [torch.zeros(shape, dtype=torch.int16).pin_memory() for _ in range(w.L)]
+        ovb = [torch.zeros(shape, dtype=torch.int16).pin_memory() for _ in range(w.L)]
+        counts = np.zeros((w.Bt, w.L), dtype=np.int32)
+        for _ in range(2):                              # the second call reuses the staging buffers
+            B.dkv_run_prefill_pass_host(g.h, hq, hk, hv, okb, ovb, counts)
+            assert (counts == g.counts).all()
+            for l in range(w.L):
+                n = int(counts[0, l]) + w.ws
+                assert torch.equal(okb[l][:, :, :n], g.kb[l].cpu()[:, :, :n])
+                assert torch.equal(ovb[l][:, :, :n], g.vb[l].cpu()[:, :, :n])
+    finally:
+        g.close()
