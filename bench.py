@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Benchmark of the DynamicKV compression pass: prefix tokens/s through all layers.
+
+One step = one whole pass of Algorithm 1 (score, per-head top-k, gather for every layer; rebudget
+and shrink every m layers) over one synthetic prompt batch, through the C ABI of libdkv.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line (rank 0).  Under torchrun each rank runs an independent replica of the whole
+workload on its own GPU (the path has no cross-GPU exchange); the time is the max over ranks.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2412_14838_b200 import synth  # noqa: E402
+
+METRIC = "prefix tokens/s through 32-layer KV compression at 32K ctx; HBM GB/s vs 8 TB/s"
+UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "mistral32k"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return json.load(f), "measured"
+    except Exception:
+        return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+# ------------------------------------------------------------------------------------ CPU oracle leg
+def oracle_sample(w, layers: int, inputs=None):
+    """Time the oracle, as it stands, on the first `layers` layers of the workload.
+
+    Returns (seconds, threads used).  Input generation is outside the timed part."""
+    from oracle import dynamickv as O
+    if inputs is None:
+        inputs = [synth.layer_inputs(w, l) for l in range(layers)]
+
+    def layer_fn(l):
+        t = inputs[l]
+        return {"q": synth.bf16_bits_to_f64(t["q"]), "k": synth.bf16_bits_to_f64(t["k"]),
+                "k_rows": t["k"], "v_rows": t["v"]}
+
+    t0 = time.perf_counter()
+    O.run_prefill_pass(layer_fn, layers, ws=w.ws, pool=w.pool, N=w.N, Bl=w.Bl, m=w.m)
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    return dt, int(cores)
+
+
+def cpu_baseline(w, layers: int):
+    dt, cores = oracle_sample(w, layers)
+    value = w.Bt * w.S / (dt * w.L / layers)
+    return {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"layers 0..{layers - 1} of {w.L} (one update block) of workload {w.name}: {dt:.2f} s, "
+                      f"scaled by {w.L}/{layers} to a whole pass"}
+
+
+def run_reference(args, w):
+    # one update block per step when few steps are asked for, one layer per step otherwise,
+    # so that the whole run stays within a few minutes
+    layers = min(w.m, w.L) if args.steps <= 5 else 1
+    inputs = [synth.layer_inputs(w, l) for l in range(layers)]
+    cores = 1
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(w, layers, inputs)
+    times = []
+    for _ in range(args.steps):
+        dt, cores = oracle_sample(w, layers, inputs)
+        times.append(dt)
+    per_step = float(np.mean(times)) * w.L / layers
+    value = w.Bt * w.S / per_step
+    base = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"each step = layers 0..{layers - 1} of {w.L} of workload {w.name} "
+                      f"({float(np.mean(times)):.2f} s), scaled by {w.L}/{layers} to a whole pass"}
+    return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w), "cpu_baseline": base,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def workload_config(w):
+    return {"workload": w.name, "layers": w.L, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D, "batch": w.Bt,
+            "prefix_len": w.S, "window": w.ws, "pool": w.pool, "avg_budget": w.N, "layer_max": w.Bl,
+            "update_interval": w.m, "recipe": w.recipe, "seed": synth.BASE_SEED,
+            "l2": "inputs (K+V of all layers, %.1f GB) exceed L2; no flush needed" %
+                  (2 * w.L * w.k_bytes_per_layer() / 1e9)}
+
+
+# ------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    BAD = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown"}
+    NOTE = {0x4: "sw_power_cap"}
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz, self.err = [], set(), None, None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            p = torch.cuda.get_device_properties(device_index)
+            bus = "%08x:%02x:%02x.0" % (p.pci_domain_id, p.pci_bus_id, p.pci_device_id)
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByPciBusId(bus.encode())
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:      # NVML missing: report that instead of a number
+            self.err = repr(e)
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in {**self.BAD, **self.NOTE}.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception as e:
+                self.err = repr(e)
+                return
+            time.sleep(0.02)
+
+    def __enter__(self):
+        if self.err is None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if self.err is not None and not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "error": self.err}
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------ GPU leg
+def run_gpu(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2412_14838_b200 import binding as B
+    from paper_2412_14838_b200 import build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    B.load()
+
+    # inputs: the same seeded bits on every rank (independent replicas of one workload)
+    to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda()
+    q, k, v = [], [], []
+    want_e2e = not args.no_e2e
+    hq, hk, hv = [], [], []
+    for l in range(w.L):
+        t = synth.layer_inputs(w, l)
+        q.append(to_dev(t["q"])); k.append(to_dev(t["k"])); v.append(to_dev(t["v"]))
+        if want_e2e:
+            for dst, name in ((hq, "q"), (hk, "k"), (hv, "v")):
+                dst.append(torch.from_numpy(t[name].view(np.int16)).pin_memory())
+    shape = (w.Bt, w.Hkv, w.Blc + w.ws, w.D)
+    kb = [torch.zeros(shape, dtype=torch.int16, device="cuda") for _ in range(w.L)]
+    vb = [torch.zeros(shape, dtype=torch.int16, device="cuda") for _ in range(w.L)]
+    ctx = B.dkv_create(B.config_of(w))
+    stream = torch.cuda.current_stream()
+
+    def one_pass():
+        B.dkv_run_prefill_pass(ctx, q, k, v, kb, vb, stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_pass()
+    barrier()
+    launches0 = B.dkv_launch_count(ctx)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        ev0.record(stream)
+        for _ in range(args.steps):
+            one_pass()
+        ev1.record(stream)
+        barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = B.dkv_launch_count(ctx) - launches0
+    tmax = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    ms = float(tmax.item())
+    ms_per_step = ms / args.steps
+    tokens = w.Bt * w.S
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    # per-kernel durations: the same steps again, each step's launches bracketed by CUDA events
+    B.dkv_profile(ctx, True)
+    for _ in range(args.steps):
+        one_pass()
+    prof = B.dkv_profile_read(ctx)
+    B.dkv_profile(ctx, False)
+    peaks, peak_kind = measured_peaks()
+    peak = float(peaks["hbm_gbs"])
+    score_ms = (prof["score_stats"][0] + prof["score_emit"][0] + prof["pool"][0]) / args.steps
+    score_launch_ms = score_ms / w.L                      # one layer's scoring = one "launch" of the scoring step
+    k_bytes = w.k_bytes_per_layer()
+    achieved = k_bytes / (score_launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "window scoring (softmax statistics sweep + emit sweep + pooling), per layer",
+                "achieved": achieved, "peak": peak, "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})",
+                "unit": "GB/s", "frac": achieved / peak,
+                "algorithmic_bytes_per_launch": k_bytes, "avg_launch_ms": score_launch_ms,
+                "traffic": None,
+                "whole_pass": {"algorithmic_bytes": w.algorithmic_bytes(),
+                               "achieved_gbs": w.algorithmic_bytes() / (ms_per_step * 1e-3) / 1e9,
+                               "frac_of_measured_peak": w.algorithmic_bytes() / (ms_per_step * 1e-3) / 1e9 / peak,
+                               "frac_of_8TBs": w.algorithmic_bytes() / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
+                "step_ms_per_pass": {n: round(t / args.steps, 4) for n, (t, _) in prof.items() if t > 0}}
+
+    # end to end: host buffers in, compacted buffers + counts out, copies inside the timed region
+    e2e = None
+    if want_e2e:
+        okb = [torch.zeros(shape, dtype=torch.int16).pin_memory() for _ in range(w.L)]
+        ovb = [torch.zeros(shape, dtype=torch.int16).pin_memory() for _ in range(w.L)]
+        counts = np.zeros((w.Bt, w.L), dtype=np.int32)
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        B.dkv_run_prefill_pass_host(ctx, hq, hk, hv, okb, ovb, counts)      # warm-up (allocates staging)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            B.dkv_run_prefill_pass_host(ctx, hq, hk, hv, okb, ovb, counts)
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t0) / e2e_steps
+        tdt = torch.tensor([dt], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(tdt, op=dist.ReduceOp.MAX)
+        dt = float(tdt.item())
+        h2d = sum(t.numel() * 2 for t in hq) + sum(t.numel() * 2 for t in hk) + sum(t.numel() * 2 for t in hv)
+        d2h = sum(t.numel() * 2 for t in okb) + sum(t.numel() * 2 for t in ovb) + counts.nbytes
+        e2e = {"value": world * tokens / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+               "ms_per_step": dt * 1e3, "steps": e2e_steps, "api": "dkv_run_prefill_pass_host (pinned host buffers)"}
+
+    B.dkv_destroy(ctx)
+    out = None
+    if rank == 0:
+        base = None
+        if world == 1 and not args.no_cpu_baseline:
+            base = cpu_baseline(w, min(w.m, w.L))
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+               "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
+               "config": dict(workload_config(w), parallelism=f"{world} independent replica(s)"),
+               "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+               "cpu_baseline": base}
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="dkv", choices=["dkv", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) != 0:
+            return 0
+        print(json.dumps(run_reference(args, w)))
+        return 0
+    if args.warmup < 3:
+        args.warmup = 3
+    out = run_gpu(args, w)
+    if out is not None:
+        print(json.dumps(out))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -143,6 +143,20 @@ int dkv_memcpy_to_host(dkv_ctx* ctx, void* host_dst, const void* dev_src, uint64
 /* Copy the status words to host int32 [8] (synchronises the device):
  * [0] first device-side error (0 = none), [1] kernels launched since dkv_create (host counter). */
 int dkv_last_status(dkv_ctx* ctx, int32_t* host_status);
+/* Optional per-step timing.  While enabled, every step's launches are bracketed by a pair of CUDA
+ * events on the step's stream.  dkv_profile_read synchronises the device and returns, per step
+ * (DKV_STEP_*), the summed event time in milliseconds and the number of kernels covered since the
+ * last read, then clears the sums.  ms, launches : host arrays of DKV_N_STEPS entries. */
+#define DKV_STEP_SCORE_STATS 0   /* sweep 1 of the scoring: softmax statistics per window row */
+#define DKV_STEP_SCORE_EMIT  1   /* sweep 2 of the scoring: per-token sums                    */
+#define DKV_STEP_POOL        2
+#define DKV_STEP_SELECT      3
+#define DKV_STEP_GATHER      4
+#define DKV_STEP_REBUDGET    5
+#define DKV_STEP_SHRINK      6
+#define DKV_N_STEPS          8
+int dkv_profile(dkv_ctx* ctx, int enable);
+int dkv_profile_read(dkv_ctx* ctx, double* ms, int64_t* launches);
 /* Kernels this context has launched since dkv_create (host counter, no synchronisation); -1 if ctx is NULL. */
 int64_t dkv_launch_count(dkv_ctx* ctx);
 /* CUDA error code of the last DKV_ERR_CUDA on this context (0 = none). */

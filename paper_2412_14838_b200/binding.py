@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(HERE, "libdkv.so")
 EXPORTS = [
     "dkv_create", "dkv_destroy", "dkv_reset", "dkv_score", "dkv_set_scores", "dkv_select_topk", "dkv_rebudget",
     "dkv_compact", "dkv_compact_all", "dkv_run_prefill_pass", "dkv_run_prefill_pass_host", "dkv_get_counts",
-    "dkv_layer_views", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status", "dkv_launch_count", "dkv_last_cuda_error",
+    "dkv_layer_views", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status", "dkv_profile", "dkv_profile_read", "dkv_launch_count", "dkv_last_cuda_error",
     "dkv_strerror", "dkv_version",
 ]
 
@@ -66,6 +66,8 @@ def load() -> ctypes.CDLL:
         "dkv_budget_views": [vp, pp, pp, pp, pp],
         "dkv_memcpy_to_host": [vp, vp, vp, ctypes.c_uint64, vp],
         "dkv_last_status": [vp, vp],
+        "dkv_profile": [vp, ctypes.c_int],
+        "dkv_profile_read": [vp, vp, vp],
         "dkv_last_cuda_error": [vp],
         "dkv_strerror": [ctypes.c_int],
         "dkv_version": [],
@@ -219,6 +221,21 @@ def dkv_last_status(ctx: int):
     buf = (ctypes.c_int32 * 8)()
     code = load().dkv_last_status(ctx, buf)
     return code, list(buf)
+
+
+STEP_NAMES = ["score_stats", "score_emit", "pool", "select", "gather", "rebudget", "shrink", "other"]
+
+
+def dkv_profile(ctx: int, enable: bool) -> None:
+    _check(load().dkv_profile(ctx, int(enable)), "dkv_profile")
+
+
+def dkv_profile_read(ctx: int):
+    """{step name: (milliseconds, kernels)} accumulated since the last read."""
+    ms = (ctypes.c_double * 8)()
+    n = (ctypes.c_int64 * 8)()
+    _check(load().dkv_profile_read(ctx, ms, n), "dkv_profile_read")
+    return {STEP_NAMES[i]: (ms[i], int(n[i])) for i in range(8)}
 
 
 def dkv_launch_count(ctx: int) -> int:

@@ -5,6 +5,7 @@
 #include <stdlib.h>
 #include <string.h>
 #include <new>
+#include <vector>
 
 #include "../../include/dkv.h"
 #include "common.cuh"
@@ -14,6 +15,8 @@
 #include "select.cuh"
 
 using namespace dkv;
+
+struct ProfRec { cudaEvent_t a, b; int step; int launches; };
 
 struct dkv_ctx {
   dkv_config cfg;
@@ -39,6 +42,12 @@ struct dkv_ctx {
   uint8_t scored[DKV_MAX_LAYERS], selected[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
   long long launches;
   int last_cuda;
+  // optional per-step timing with CUDA events (dkv_profile)
+  bool prof_on;
+  std::vector<ProfRec>* prof_recs;
+  size_t prof_used;
+  double prof_ms[DKV_N_STEPS];
+  long long prof_launches[DKV_N_STEPS];
   // staging for the host-buffer pass (allocated on first use)
   bool staged;
   void *st_q[2], *st_k[2], *st_v[2];
@@ -67,6 +76,23 @@ int cuda_fail(dkv_ctx* c, cudaError_t e) {
     cudaError_t e__ = cudaPeekAtLastError();                  \
     if (e__ != cudaSuccess) return cuda_fail((ctx), e__);     \
   } while (0)
+
+// Event pair around one step's launches; read back by dkv_profile_read.
+struct ProfScope {
+  dkv_ctx* c; cudaStream_t st; ProfRec* r;
+  ProfScope(dkv_ctx* c_, int step, int launches, cudaStream_t st_) : c(c_), st(st_), r(nullptr) {
+    if (!c->prof_on) return;
+    if (c->prof_used == c->prof_recs->size()) {
+      ProfRec n; n.step = 0; n.launches = 0;
+      if (cudaEventCreate(&n.a) != cudaSuccess || cudaEventCreate(&n.b) != cudaSuccess) return;
+      c->prof_recs->push_back(n);
+    }
+    r = &(*c->prof_recs)[c->prof_used++];
+    r->step = step; r->launches = launches;
+    cudaEventRecord(r->a, st);
+  }
+  ~ProfScope() { if (r) cudaEventRecord(r->b, st); }
+};
 
 size_t layer_scores(const Shape& s) { return (size_t)s.Bt * s.Hkv * s.P; }
 size_t layer_idx(const Shape& s) { return (size_t)s.Bt * s.Hkv * s.Blc; }
@@ -103,18 +129,24 @@ int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_
   const uint16_t* kp = static_cast<const uint16_t*>(k);
   const dim3 g1(c->n_split, s.Bt * s.Hkv), g2(c->emit_ctas, s.Bt * s.Hkv);
   const int threads = c->m_stride;
-  if (s.D == 128) {
-    score_stats_simt<128><<<g1, threads, 0, st>>>(qp, kp, c->d_stats, s, c->keys_per_split, c->n_split, c->m_stride);
+  {
+    ProfScope ps(c, DKV_STEP_SCORE_STATS, 1, st);
+    if (s.D == 128)
+      score_stats_simt<128><<<g1, threads, 0, st>>>(qp, kp, c->d_stats, s, c->keys_per_split, c->n_split, c->m_stride);
+    else
+      score_stats_simt<64><<<g1, threads, 0, st>>>(qp, kp, c->d_stats, s, c->keys_per_split, c->n_split, c->m_stride);
     DKV_LAUNCHED(c);
-    score_emit_simt<128><<<g2, threads, 0, st>>>(qp, kp, c->d_stats, c->d_raw, s, c->keys_per_emit, c->n_split, c->m_stride);
-    DKV_LAUNCHED(c);
-  } else {
-    score_stats_simt<64><<<g1, threads, 0, st>>>(qp, kp, c->d_stats, s, c->keys_per_split, c->n_split, c->m_stride);
-    DKV_LAUNCHED(c);
-    score_emit_simt<64><<<g2, threads, 0, st>>>(qp, kp, c->d_stats, c->d_raw, s, c->keys_per_emit, c->n_split, c->m_stride);
+  }
+  {
+    ProfScope ps(c, DKV_STEP_SCORE_EMIT, 1, st);
+    if (s.D == 128)
+      score_emit_simt<128><<<g2, threads, 0, st>>>(qp, kp, c->d_stats, c->d_raw, s, c->keys_per_emit, c->n_split, c->m_stride);
+    else
+      score_emit_simt<64><<<g2, threads, 0, st>>>(qp, kp, c->d_stats, c->d_raw, s, c->keys_per_emit, c->n_split, c->m_stride);
     DKV_LAUNCHED(c);
   }
   const size_t total = layer_scores(s);
+  ProfScope ps(c, DKV_STEP_POOL, 1, st);
   maxpool_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(c->d_raw, c->d_scores + (size_t)layer * total, scores_out,
                                                                   s.P, s.pool / 2, total);
   DKV_LAUNCHED(c);
@@ -126,6 +158,7 @@ int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_
 // ---- step (2): per-head top-Bl' ----------------------------------------------------------------
 int do_select(dkv_ctx* c, int layer, int* idx_out, int* rank_out, cudaStream_t st) {
   const Shape& s = c->s;
+  ProfScope ps(c, DKV_STEP_SELECT, 1, st);
   select_topk_kernel<<<s.Bt * s.Hkv, kSelThreads, (size_t)c->sort_n * 8, st>>>(
       c->d_scores + (size_t)layer * layer_scores(s), c->d_idx + (size_t)layer * layer_idx(s),
       c->d_rank + (size_t)layer * layer_idx(s), idx_out, rank_out, s.P, s.Blc, c->sort_n, c->d_count, s.Hkv, s.L, layer);
@@ -142,6 +175,7 @@ int do_rebudget(dkv_ctx* c, int l, int* counts_out, cudaStream_t st) {
   long long k = (long long)s.N * s.Hkv * l;
   const long long pop = (long long)l * (long long)per_layer;
   if (k > pop) k = pop;
+  ProfScope ps(c, DKV_STEP_REBUDGET, 9, st);
   const int init_n = 3 * s.Bt * kRbBins > s.Bt * s.L ? 3 * s.Bt * kRbBins : s.Bt * s.L;
   rb_init_kernel<<<(init_n + 255) / 256, 256, 0, st>>>(c->d_rb_state, c->d_rb_hist, c->d_cnt_gt, c->d_cnt_eq, s.Bt, s.L,
                                                       (unsigned int)k);
@@ -171,6 +205,7 @@ int do_shrink(dkv_ctx* c, int layer0, int n, void* const* kb, void* const* vb, c
   const Shape& s = c->s;
   LayerPtrs ptrs;
   for (int i = 0; i < n; ++i) { ptrs.kb[layer0 + i] = kb[i]; ptrs.vb[layer0 + i] = vb[i]; }
+  ProfScope ps(c, DKV_STEP_SHRINK, 2, st);
   shrink_kernel<<<dim3(s.Bt * s.Hkv, n), kShrinkThreads, (size_t)s.Blc * 4, st>>>(
       ptrs, layer0, c->d_idx, c->d_rank, c->d_count, c->d_held, s.Bt, s.Hkv, s.L, s.ws, s.Blc, s.rows, s.D * 2 / 16,
       layer_idx(s));
@@ -184,11 +219,14 @@ int do_gather(dkv_ctx* c, int layer, const void* k_src, const void* v_src, void*
   const Shape& s = c->s;
   const int vec = s.D * 2 / 16, rpb = 256 / vec;
   const dim3 grid((s.rows + rpb - 1) / rpb, s.Bt * s.Hkv, 2);
+  {
+  ProfScope ps(c, DKV_STEP_GATHER, 1, st);
   gather_rows_kernel<<<grid, 256, 0, st>>>(static_cast<const uint4*>(k_src), static_cast<const uint4*>(v_src),
                                            static_cast<uint4*>(kb), static_cast<uint4*>(vb),
                                            c->d_idx + (size_t)layer * layer_idx(s), s.Blc, s.S, s.P, s.ws, s.rows, vec,
                                            c->d_held, s.Hkv, s.L, layer);
   DKV_LAUNCHED(c);
+  }
   c->gathered[layer] = 1;
   if (c->stale[layer]) {           // an update ran between select and gather: apply it now
     c->stale[layer] = 0;
@@ -231,6 +269,10 @@ void free_all(dkv_ctx* c) {
   cudaFree(c->d_scores); cudaFree(c->d_raw); cudaFree(c->d_idx); cudaFree(c->d_rank); cudaFree(c->d_count);
   cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_stats); cudaFree(c->d_rb_state); cudaFree(c->d_rb_hist);
   cudaFree(c->d_cnt_gt); cudaFree(c->d_cnt_eq); cudaFree(c->d_status);
+  if (c->prof_recs) {
+    for (ProfRec& r : *c->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    delete c->prof_recs;
+  }
   if (c->staged) {
     for (int i = 0; i < 2; ++i) {
       cudaFree(c->st_q[i]); cudaFree(c->st_k[i]); cudaFree(c->st_v[i]);
@@ -289,6 +331,8 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   if (!c) return DKV_ERR_NOMEM;
   memset(c, 0, sizeof *c);
   c->cfg = *cfg;
+  c->prof_recs = new (std::nothrow) std::vector<ProfRec>();
+  if (!c->prof_recs) { delete c; return DKV_ERR_NOMEM; }
   Shape& s = c->s;
   s.L = cfg->n_layers; s.Hq = cfg->n_q_heads; s.Hkv = cfg->n_kv_heads; s.D = cfg->head_dim; s.Bt = cfg->batch;
   s.S = cfg->seq_len; s.ws = cfg->window; s.pool = cfg->pool_kernel; s.N = cfg->avg_budget; s.Bl = cfg->layer_max;
@@ -509,6 +553,31 @@ int dkv_last_status(dkv_ctx* c, int32_t* host_status) {
   DKV_CUDA(c, cudaMemcpy(host_status, c->d_status, sizeof(int) * 8, cudaMemcpyDeviceToHost));
   host_status[1] = (int32_t)(c->launches & 0x7FFFFFFF);
   return host_status[0] == 0 ? DKV_OK : host_status[0];
+}
+
+int dkv_profile(dkv_ctx* c, int enable) {
+  if (!c) return DKV_ERR_INVALID_ARG;
+  c->prof_on = enable != 0;
+  return DKV_OK;
+}
+
+int dkv_profile_read(dkv_ctx* c, double* ms, int64_t* launches) {
+  if (!c || !ms || !launches) return DKV_ERR_INVALID_ARG;
+  DKV_CUDA(c, cudaDeviceSynchronize());
+  for (size_t i = 0; i < c->prof_used; ++i) {
+    const ProfRec& r = (*c->prof_recs)[i];
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, r.a, r.b) == cudaSuccess) {
+      c->prof_ms[r.step] += t;
+      c->prof_launches[r.step] += r.launches;
+    }
+  }
+  c->prof_used = 0;
+  for (int i = 0; i < DKV_N_STEPS; ++i) {
+    ms[i] = c->prof_ms[i]; launches[i] = c->prof_launches[i];
+    c->prof_ms[i] = 0; c->prof_launches[i] = 0;
+  }
+  return DKV_OK;
 }
 
 int64_t dkv_launch_count(dkv_ctx* c) { return c ? (int64_t)c->launches : -1; }
