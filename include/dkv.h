@@ -55,7 +55,7 @@ typedef struct {
   int32_t batch;            /* Bt                                                                 */
   int32_t seq_len;          /* S   : includes the window; S > ws                                  */
   int32_t window;           /* ws  : ws * G <= DKV_MAX_WINDOW_ROWS                                */
-  int32_t pool_kernel;      /* odd width of the 1-D pooling of Eq. 2, >= 1                        */
+  int32_t pool_kernel;      /* odd width of the 1-D pooling of Eq. 2, 1..255                      */
   int32_t pool_kind;        /* 0 = max-pool (only kind built)                                     */
   int32_t avg_budget;       /* N = wt - ws : retained prefix tokens per head per layer on average */
   int32_t layer_max;        /* Bl = floor(N * r_max), N <= Bl <= DKV_MAX_LAYER_BUDGET             */

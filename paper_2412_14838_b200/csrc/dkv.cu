@@ -12,6 +12,7 @@
 #include "compact.cuh"
 #include "rebudget.cuh"
 #include "score_simt.cuh"
+#include "score_tc.cuh"
 #include "select.cuh"
 
 using namespace dkv;
@@ -38,6 +39,10 @@ struct dkv_ctx {
   int* d_status;        // [8]
   int n_split, keys_per_split, m_stride, emit_ctas, keys_per_emit;
   int sort_n;
+  // tensor-core scoring
+  bool use_simt;
+  int n_sms, tc_stats_grid, tc_emit_grid, tc_slots;
+  float2* d_tc_stats;   // [Bt*Hkv][tc_slots][256]
   // host state
   uint8_t scored[DKV_MAX_LAYERS], selected[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
   long long launches;
@@ -106,6 +111,7 @@ int validate(const dkv_config* c) {
   if (c->n_q_heads % c->n_kv_heads != 0) return DKV_ERR_INVALID_ARG;
   if (c->window < 1 || c->seq_len <= c->window) return DKV_ERR_INVALID_ARG;
   if (c->pool_kernel < 1 || c->pool_kernel % 2 == 0) return DKV_ERR_INVALID_ARG;
+  if (c->pool_kernel > 255) return DKV_ERR_UNSUPPORTED;
   if (c->avg_budget < 1 || c->layer_max < c->avg_budget || c->update_interval < 1) return DKV_ERR_INVALID_ARG;
   if (c->flags != 0) return DKV_ERR_INVALID_ARG;
   if (c->pool_kind != 0) return DKV_ERR_UNSUPPORTED;
@@ -123,7 +129,76 @@ int check_layer(const dkv_ctx* c, int layer) {
 }
 
 // ---- step (1): scores of one layer -------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor [heads][rows][D] seen as (D, rows, heads); boxes of 64 columns x 128 rows, 128-byte swizzle,
+// rows past the end of a head read as zero.
+bool make_map(CUtensorMap* m, const void* base, int D, int rows, int heads) {
+  EncodeTiledFn fn = encode_tiled();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)heads};
+  const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)rows * D * 2};
+  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+uint32_t make_idesc(int M, int N) {
+  // fp32 accumulator, bf16 A and B, both K-major
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+int do_score_tc(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
+  const Shape& s = c->s;
+  const int heads = s.Bt * s.Hkv;
+  CUtensorMap qm, km;
+  if (!make_map(&qm, q, s.D, s.M, heads) || !make_map(&km, k, s.D, s.S, heads)) return DKV_ERR_CUDA;
+  tc::Params p;
+  p.S = s.S; p.P = s.P; p.ws = s.ws; p.M = s.M; p.D = s.D; p.heads = heads; p.half = s.pool / 2;
+  p.tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
+  p.nq16 = (s.M + 15) / 16 * 16;
+  p.nmblk = (s.M + 127) / 128;
+  p.slots = c->tc_slots; p.m_stride = 256;
+  p.scale2 = kLog2e / sqrtf((float)s.D);
+  p.stats = c->d_tc_stats;
+  p.scores = c->d_scores + (size_t)layer * layer_scores(s);
+  p.copy_out = scores_out;
+  p.status = c->d_status;
+  {
+    ProfScope ps(c, DKV_STEP_SCORE_STATS, 1, st);
+    p.idesc = make_idesc(128, 128);
+    tc::score_tc_kernel<tc::kStats><<<c->tc_stats_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, p, c->tc_stats_grid);
+    DKV_LAUNCHED(c);
+  }
+  {
+    ProfScope ps(c, DKV_STEP_SCORE_EMIT, 1, st);
+    p.idesc = make_idesc(128, p.nq16);
+    tc::score_tc_kernel<tc::kEmit><<<c->tc_emit_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, p, c->tc_stats_grid);
+    DKV_LAUNCHED(c);
+  }
+  c->scored[layer] = 1;
+  c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
+  return DKV_OK;
+}
+
 int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
+  if (!c->use_simt) return do_score_tc(c, layer, q, k, scores_out, st);
   const Shape& s = c->s;
   const uint16_t* qp = static_cast<const uint16_t*>(q);
   const uint16_t* kp = static_cast<const uint16_t*>(k);
@@ -268,7 +343,7 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
 void free_all(dkv_ctx* c) {
   cudaFree(c->d_scores); cudaFree(c->d_raw); cudaFree(c->d_idx); cudaFree(c->d_rank); cudaFree(c->d_count);
   cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_stats); cudaFree(c->d_rb_state); cudaFree(c->d_rb_hist);
-  cudaFree(c->d_cnt_gt); cudaFree(c->d_cnt_eq); cudaFree(c->d_status);
+  cudaFree(c->d_cnt_gt); cudaFree(c->d_cnt_eq); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
   if (c->prof_recs) {
     for (ProfRec& r : *c->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     delete c->prof_recs;
@@ -352,6 +427,25 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   while (c->sort_n < s.Blc) c->sort_n <<= 1;
 
   cudaError_t e = cudaGetDevice(&c->device);
+  {
+    const char* impl = getenv("DKV_SCORE_IMPL");
+    c->use_simt = impl && strcmp(impl, "simt") == 0;
+    int sms = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
+    c->n_sms = sms > 0 ? sms : 1;
+    const int tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
+    const long long total_tiles = (long long)heads * tph;
+    c->tc_stats_grid = (int)(total_tiles < c->n_sms ? total_tiles : c->n_sms);
+    const long long out_tiles = ((long long)heads * s.P + tc::kTileKeys - 1) / tc::kTileKeys;
+    c->tc_emit_grid = (int)(out_tiles < c->n_sms ? out_tiles : c->n_sms);
+    int slots = 1;
+    for (int bh = 0; bh < heads; ++bh) {
+      const int lo = tc::tile_owner((long long)bh * tph, total_tiles, c->tc_stats_grid);
+      const int hi = tc::tile_owner((long long)(bh + 1) * tph - 1, total_tiles, c->tc_stats_grid);
+      if (hi - lo + 1 > slots) slots = hi - lo + 1;
+    }
+    c->tc_slots = slots;
+  }
   const size_t bl = (size_t)s.Bt * s.L;
 #define TRY(call) if (e == cudaSuccess) e = (call)
   TRY(cudaMalloc(&c->d_scores, sizeof(float) * s.L * layer_scores(s)));
@@ -366,6 +460,9 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMalloc(&c->d_rb_hist, sizeof(unsigned int) * 3 * s.Bt * kRbBins));
   TRY(cudaMalloc(&c->d_cnt_gt, sizeof(unsigned int) * bl));
   TRY(cudaMalloc(&c->d_cnt_eq, sizeof(unsigned int) * bl));
+  TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * heads * c->tc_slots * 256));
+  TRY(cudaFuncSetAttribute(tc::score_tc_kernel<tc::kStats>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  TRY(cudaFuncSetAttribute(tc::score_tc_kernel<tc::kEmit>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   TRY(cudaMalloc(&c->d_status, sizeof(int) * 8));
   TRY(cudaMemset(c->d_status, 0, sizeof(int) * 8));
   TRY(cudaMemset(c->d_count, 0, sizeof(int) * bl));

@@ -1,0 +1,438 @@
+// Window scoring (Eq. 1-2, Algorithm 1's scoring line) on the sm_100a tensor cores.
+//
+// A token's score needs the softmax normaliser of every window row, which is only known after
+// all keys have been seen, so the keys are swept twice:
+//   sweep 1 (kStats)  logits = Q_win . K^T, one TMEM lane per window row; every thread keeps the
+//                     running (max, sum) of its own row over the CTA's key range;
+//   sweep 2 (kEmit)   logits^T = K . Q_win^T, one TMEM lane per KEY; every thread adds up
+//                     2^(logit - lse_row) over the rows of its own key, which is the token's score
+//                     with no cross-thread reduction; the CTA then max-pools its key range.
+// Both sweeps share one pipeline: a TMA producer warp streams 128-key tiles of K (bf16, 128-byte
+// swizzle) through a shared-memory ring, one thread issues tcgen05.mma into double-buffered TMEM
+// accumulators, and two groups of four warps read the accumulators back with tcgen05.ld.
+// Work is split evenly: the flattened (head, key tile) space for sweep 1 and the flattened
+// (head, prefix position) space for sweep 2 are cut into one contiguous slice per CTA.
+#pragma once
+#include <cuda.h>
+#include "common.cuh"
+
+namespace dkv {
+namespace tc {
+
+constexpr int kTileKeys = 128;
+constexpr int kStages = 4;                 // K tiles in flight
+constexpr int kThreads = 320;              // warp 0: TMA, warp 1: MMA, warps 2..9: two softmax groups
+constexpr int kSoftmaxThreads = 256;
+constexpr int kMaxSegTiles = 16;           // sweep 2: tiles per pooled segment
+constexpr int kHalfBytes = 128 * 128;      // one 128-row x 64-column bf16 box
+constexpr int kQRegion = 2 * 2 * kHalfBytes;          // up to 256 rows x 128 columns
+constexpr int kKRegion = kStages * 2 * kHalfBytes;    // ring of 128 x 128 tiles
+constexpr int kSmemBytes = 1024 /*align*/ + kQRegion + kKRegion + 4096 /*lse, merge*/ +
+                           kMaxSegTiles * kTileKeys * 4 /*raw*/ + 256 /*barriers*/;
+constexpr long long kWaitCycles = 4000000000ll;       // ~2 s: a wait that long is reported, not spun on
+
+enum Mode { kStats = 0, kEmit = 1 };
+
+struct Params {
+  int S, P, ws, M, D, heads, half;
+  int tph;                 // key tiles per head, ceil(S / 128)
+  int nq16;                // window rows rounded up to 16 (MMA N of sweep 2)
+  int nmblk;               // 128-row blocks of window rows (MMA M blocks of sweep 1)
+  int slots;               // partial-statistics slots per head
+  int m_stride;            // floats2 per slot
+  float scale2;            // log2(e) / sqrt(D)
+  uint32_t idesc;          // tcgen05 instruction descriptor of this sweep
+  float2* stats;
+  float* scores;           // [heads][P] pooled scores (sweep 2)
+  float* copy_out;         // optional second copy
+  int* status;             // device status words; [0] = first error
+};
+
+// ------------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after kWaitCycles, records the failure and lets the kernel run to its end.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+  if (*abort_flag) return;
+  if (mbar_try(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!mbar_try(bar, parity)) {
+    if (*abort_flag) return;
+    if (clock64() - t0 > kWaitCycles) {
+      *abort_flag = 1;
+      atomicCAS(status, 0, code);
+      return;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor: K-major, 128-byte swizzle, rows 128 B apart, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address
+  d |= (uint64_t)1 << 16;                            // leading byte offset (unused with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset
+  d |= (uint64_t)1 << 46;                            // descriptor version of sm_100
+  d |= (uint64_t)2 << 61;                            // 128-byte swizzle
+  return d;
+}
+
+// ------------------------------------------------------------------------------------------ work split
+struct Seg {
+  int bh;        // head (sample * Hkv + kv head)
+  int key0;      // first key of the first tile (may be negative in sweep 2: the pooling halo)
+  int ntiles;
+  int out0, out1;  // sweep 2: prefix positions this segment writes
+  bool new_head;
+};
+
+template <int MODE>
+struct SegIter {
+  long long u, u_end;
+  int uph, half, cur_bh;
+  __device__ SegIter(const Params& p, int cta, int grid) {
+    uph = MODE == kStats ? p.tph : p.P;
+    const long long total = (long long)p.heads * uph;
+    u = total * cta / grid;
+    u_end = total * (cta + 1) / grid;
+    half = p.half;
+    cur_bh = -1;
+  }
+  __device__ bool next(Seg& s) {
+    if (u >= u_end) return false;
+    const int bh = (int)(u / uph), off = (int)(u % uph);
+    long long e = (long long)(bh + 1) * uph;
+    if (e > u_end) e = u_end;
+    if (MODE == kEmit && e > u + (kMaxSegTiles * kTileKeys - 2 * half)) e = u + (kMaxSegTiles * kTileKeys - 2 * half);
+    const int len = (int)(e - u);
+    s.bh = bh;
+    if (MODE == kStats) {
+      s.key0 = off * kTileKeys; s.ntiles = len; s.out0 = s.out1 = 0;
+    } else {
+      s.out0 = off; s.out1 = off + len; s.key0 = off - half;
+      s.ntiles = (len + 2 * half + kTileKeys - 1) / kTileKeys;
+    }
+    s.new_head = bh != cur_bh;
+    cur_bh = bh;
+    u = e;
+    return true;
+  }
+};
+
+// CTA that owns key tile x of the flattened (head, tile) space, when `total` tiles are cut into `grid` slices.
+__host__ __device__ __forceinline__ int tile_owner(long long x, long long total, int grid) {
+  return (int)(((x + 1) * grid + total - 1) / total) - 1;
+}
+
+// ------------------------------------------------------------------------------------------ kernel
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map, const Params p,
+                int stats_grid) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* q_smem = smem;                              // [half][256 rows][128 B]
+  uint8_t* k_smem = smem + kQRegion;                   // [stage][half][128 rows][128 B]
+  float* lse_s = reinterpret_cast<float*>(k_smem + kKRegion);          // [256] lse2 per window row (sweep 2)
+  float2* merge_s = reinterpret_cast<float2*>(lse_s + 256);            // [256] group-B partials (sweep 1)
+  float* raw_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(lse_s) + 4096);   // [16 * 128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(raw_s + kMaxSegTiles * kTileKeys);
+  // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2], q_full
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+  const uint32_t bar0 = smem_u32(bars);
+  auto FULL = [&](int s) { return bar0 + 8u * s; };
+  auto EMPTY = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto TFULL = [&](int t) { return bar0 + 8u * (2 * kStages + t); };
+  auto TEMPTY = [&](int t) { return bar0 + 8u * (2 * kStages + 2 + t); };
+  const uint32_t QFULL = bar0 + 8u * (2 * kStages + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int halves = p.D / 64;
+  const uint32_t tile_bytes = (uint32_t)halves * kHalfBytes;
+  volatile int* abort_flag = &abort_s;
+
+  if (threadIdx.x == 0) {
+    abort_s = 0;
+    for (int s = 0; s < kStages; ++s) { mbar_init(FULL(s), 1); mbar_init(EMPTY(s), 1); }
+    for (int t = 0; t < 2; ++t) { mbar_init(TFULL(t), 1); mbar_init(TEMPTY(t), 4); }
+    mbar_init(QFULL, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+  const int stage_cols = MODE == kStats ? p.nmblk * 128 : 256;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      SegIter<MODE> it(p, blockIdx.x, gridDim.x);
+      Seg sg;
+      int tile = 0, nq = 0;
+      while (it.next(sg)) {
+        if (sg.new_head) {
+          if (tile > 0) {   // all MMAs that read the previous head's queries must have finished
+            const int last = tile - 1;
+            mbar_wait(EMPTY(last % kStages), (last / kStages) & 1, abort_flag, p.status, 101);
+          }
+          if (!*abort_flag) {
+            mbar_expect_tx(QFULL, (uint32_t)(p.nmblk * halves) * kHalfBytes);
+            for (int h = 0; h < halves; ++h)
+              for (int mb = 0; mb < p.nmblk; ++mb)
+                tma_load_3d(smem_u32(q_smem + h * (2 * kHalfBytes) + mb * kHalfBytes), &q_map, QFULL, 64 * h, 128 * mb, sg.bh);
+          }
+          ++nq;
+        }
+        for (int i = 0; i < sg.ntiles; ++i, ++tile) {
+          const int s = tile % kStages, n = tile / kStages;
+          mbar_wait(EMPTY(s), (n & 1) ^ 1, abort_flag, p.status, 102);
+          if (*abort_flag) break;
+          mbar_expect_tx(FULL(s), tile_bytes);
+          for (int h = 0; h < halves; ++h)
+            tma_load_3d(smem_u32(k_smem + (s * 2 + h) * kHalfBytes), &k_map, FULL(s), 64 * h, sg.key0 + i * kTileKeys, sg.bh);
+        }
+        if (*abort_flag) break;
+      }
+      (void)nq;
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      SegIter<MODE> it(p, blockIdx.x, gridDim.x);
+      Seg sg;
+      int tile = 0, nq = 0;
+      const int ksteps = p.D / 16;
+      while (it.next(sg)) {
+        if (sg.new_head) { mbar_wait(QFULL, nq & 1, abort_flag, p.status, 103); ++nq; }
+        for (int i = 0; i < sg.ntiles; ++i, ++tile) {
+          const int s = tile % kStages, n = tile / kStages, t = tile & 1, nt = tile >> 1;
+          mbar_wait(FULL(s), n & 1, abort_flag, p.status, 104);
+          mbar_wait(TEMPTY(t), (nt & 1) ^ 1, abort_flag, p.status, 105);
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(t * stage_cols);
+          if (MODE == kStats) {
+            for (int mb = 0; mb < p.nmblk; ++mb)
+              for (int ks = 0; ks < ksteps; ++ks) {
+                const uint64_t a = smem_desc(smem_u32(q_smem + (ks >> 2) * (2 * kHalfBytes) + mb * kHalfBytes) + (ks & 3) * 32);
+                const uint64_t b = smem_desc(smem_u32(k_smem + (s * 2 + (ks >> 2)) * kHalfBytes) + (ks & 3) * 32);
+                tc_mma(d_tmem + mb * 128, a, b, p.idesc, ks > 0);
+              }
+          } else {
+            for (int ks = 0; ks < ksteps; ++ks) {
+              const uint64_t a = smem_desc(smem_u32(k_smem + (s * 2 + (ks >> 2)) * kHalfBytes) + (ks & 3) * 32);
+              const uint64_t b = smem_desc(smem_u32(q_smem + (ks >> 2) * (2 * kHalfBytes)) + (ks & 3) * 32);
+              tc_mma(d_tmem, a, b, p.idesc, ks > 0);
+            }
+          }
+          tc_commit(EMPTY(s));      // the K slot may be refilled once these MMAs have read it
+          tc_commit(TFULL(t));      // the accumulator is complete
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax warps
+    const int sw = warp - 2;                   // 0..7
+    const int grp = sw >> 2;                   // group 0 takes even tiles, group 1 odd tiles
+    const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+    const int row = quad * 32 + lane;          // TMEM lane = window row (sweep 1) or key within the tile (sweep 2)
+    const int sid = threadIdx.x - 64;          // 0..255 among the softmax threads
+    SegIter<MODE> it(p, blockIdx.x, gridDim.x);
+    Seg sg;
+    int tile = 0;
+    while (it.next(sg)) {
+      if (MODE == kStats) {
+        float mx[2] = {-INFINITY, -INFINITY}, sum[2] = {0.f, 0.f};
+        int limit[2];
+#pragma unroll
+        for (int mb = 0; mb < 2; ++mb) limit[mb] = p.P + ((row + 128 * mb) % p.ws);
+        for (int i = 0; i < sg.ntiles; ++i, ++tile) {
+          if ((tile & 1) != grp) continue;
+          const int t = tile & 1, nt = tile >> 1;
+          mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 106);
+          tc_fence_after();
+          const int kb = sg.key0 + i * kTileKeys;
+          const bool need_mask = kb + kTileKeys - 1 > p.P;
+#pragma unroll
+          for (int mb = 0; mb < 2; ++mb) {
+            if (mb >= p.nmblk) break;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * stage_cols + mb * 128);
+#pragma unroll 1
+            for (int c = 0; c < 8; ++c) {
+              float x[16];
+              tc_ld16(taddr + c * 16, x);
+              tc_wait_ld();
+              if (need_mask) {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) if (kb + c * 16 + e > limit[mb]) x[e] = -INFINITY;
+              }
+              float cm = x[0];
+#pragma unroll
+              for (int e = 1; e < 16; ++e) cm = fmaxf(cm, x[e]);
+              if (cm == -INFINITY) continue;
+              const float mnew = fmaxf(mx[mb], cm * p.scale2);
+              if (mnew > mx[mb]) { sum[mb] *= fast_exp2(mx[mb] - mnew); mx[mb] = mnew; }
+              float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+              const float neg = -mx[mb];
+#pragma unroll
+              for (int e = 0; e < 16; e += 4) {
+                s0 += fast_exp2(fmaf(x[e], p.scale2, neg));
+                s1 += fast_exp2(fmaf(x[e + 1], p.scale2, neg));
+                s2 += fast_exp2(fmaf(x[e + 2], p.scale2, neg));
+                s3 += fast_exp2(fmaf(x[e + 3], p.scale2, neg));
+              }
+              sum[mb] += (s0 + s1) + (s2 + s3);
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(TEMPTY(t));
+        }
+        // merge the two groups' partials and publish this CTA's statistics for the head
+        if (grp == 1) {
+#pragma unroll
+          for (int mb = 0; mb < 2; ++mb) merge_s[row + 128 * mb] = make_float2(mx[mb], sum[mb]);
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (grp == 0) {
+          const long long total = (long long)p.heads * p.tph;
+          const int slot = blockIdx.x - tile_owner((long long)sg.bh * p.tph, total, gridDim.x);
+#pragma unroll
+          for (int mb = 0; mb < 2; ++mb) {
+            const int r = row + 128 * mb;
+            if (mb < p.nmblk && r < p.M) {
+              const float2 o = merge_s[r];
+              const float m = fmaxf(mx[mb], o.x);
+              float l = 0.f;
+              if (m > -INFINITY) l = sum[mb] * fast_exp2(mx[mb] - m) + o.y * fast_exp2(o.x - m);
+              p.stats[((size_t)sg.bh * p.slots + slot) * p.m_stride + r] = make_float2(m, l);
+            }
+          }
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+      } else {
+        // ---------------------------------------------------------------- sweep 2
+        if (sg.new_head) {
+          // lse2 of every window row from the partial statistics of sweep 1
+          const long long total = (long long)p.heads * p.tph;
+          const int c_lo = tile_owner((long long)sg.bh * p.tph, total, stats_grid);
+          const int c_hi = tile_owner((long long)(sg.bh + 1) * p.tph - 1, total, stats_grid);
+          float lse = INFINITY;
+          if (sid < p.M) {
+            float m = -INFINITY;
+            for (int c = 0; c <= c_hi - c_lo; ++c) m = fmaxf(m, p.stats[((size_t)sg.bh * p.slots + c) * p.m_stride + sid].x);
+            float l = 0.f;
+            for (int c = 0; c <= c_hi - c_lo; ++c) {
+              const float2 st = p.stats[((size_t)sg.bh * p.slots + c) * p.m_stride + sid];
+              l += st.y * fast_exp2(st.x - m);
+            }
+            lse = m + log2f(l);
+          }
+          lse_s[sid] = lse;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        for (int i = 0; i < sg.ntiles; ++i, ++tile) {
+          if ((tile & 1) != grp) continue;
+          const int t = tile & 1, nt = tile >> 1;
+          mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 107);
+          tc_fence_after();
+          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * stage_cols);
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < p.nq16; c += 16) {
+            float x[16];
+            tc_ld16(taddr + c, x);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; e += 4) {
+              const float4 ls = *reinterpret_cast<const float4*>(&lse_s[c + e]);
+              a0 += fast_exp2(fmaf(x[e], p.scale2, -ls.x));
+              a1 += fast_exp2(fmaf(x[e + 1], p.scale2, -ls.y));
+              a2 += fast_exp2(fmaf(x[e + 2], p.scale2, -ls.z));
+              a3 += fast_exp2(fmaf(x[e + 3], p.scale2, -ls.w));
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(TEMPTY(t));
+          raw_s[i * kTileKeys + row] = (a0 + a1) + (a2 + a3);
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // Eq. 2's pooling over this segment: raw_s[x] belongs to key key0 + x
+        for (int o = sg.out0 + sid; o < sg.out1; o += kSoftmaxThreads) {
+          const int x = o - sg.key0;
+          float v = raw_s[x];
+          for (int d = 1; d <= p.half; ++d) {
+            if (o - d >= 0) v = fmaxf(v, raw_s[x - d]);
+            if (o + d < p.P) v = fmaxf(v, raw_s[x + d]);
+          }
+          const size_t at = (size_t)sg.bh * p.P + o;
+          p.scores[at] = v;
+          if (p.copy_out) p.copy_out[at] = v;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+  }
+}
+
+}  // namespace tc
+}  // namespace dkv
