@@ -149,7 +149,7 @@ int dkv_last_status(dkv_ctx* ctx, int32_t* host_status);
  * last read, then clears the sums.  ms, launches : host arrays of DKV_N_STEPS entries. */
 #define DKV_STEP_SCORE_STATS 0   /* sweep 1 of the scoring: softmax statistics per window row */
 #define DKV_STEP_SCORE_EMIT  1   /* sweep 2 of the scoring: per-token sums                    */
-#define DKV_STEP_POOL        2
+#define DKV_STEP_POOL        2   /* unused: pooling is fused into sweep 2 */
 #define DKV_STEP_SELECT      3
 #define DKV_STEP_GATHER      4
 #define DKV_STEP_REBUDGET    5

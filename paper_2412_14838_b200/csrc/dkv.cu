@@ -11,7 +11,6 @@
 #include "common.cuh"
 #include "compact.cuh"
 #include "rebudget.cuh"
-#include "score_simt.cuh"
 #include "score_tc.cuh"
 #include "select.cuh"
 
@@ -25,22 +24,18 @@ struct dkv_ctx {
   int device;
   // device state
   float* d_scores;      // [L][Bt][Hkv][P]  pooled scores, the history A^b
-  float* d_raw;         // [Bt][Hkv][P]     un-pooled scores of the layer being scored
   int* d_idx;           // [L][Bt][Hkv][Blc] kept positions, ascending
   int* d_rank;          // [L][Bt][Hkv][Blc] their ranks
   int* d_count;         // [Bt][L] budget of each layer
   int* d_held;          // [Bt][L] rows the layer's buffers hold
   int* d_dbg;           // 3 x [Bt][L] : cnt, Z, Z' of the last update
-  float2* d_stats;      // [Bt*Hkv][n_split][m_stride] partial softmax statistics
   RbState* d_rb_state;  // [Bt]
   unsigned int* d_rb_hist;   // [3][Bt][2048]
   unsigned int* d_cnt_gt;    // [Bt][L]
   unsigned int* d_cnt_eq;    // [Bt][L]
   int* d_status;        // [8]
-  int n_split, keys_per_split, m_stride, emit_ctas, keys_per_emit;
   int sort_n;
   // tensor-core scoring
-  bool use_simt;
   int n_sms, tc_stats_grid, tc_emit_grid, tc_slots;
   float2* d_tc_stats;   // [Bt*Hkv][tc_slots][256]
   // host state
@@ -164,7 +159,7 @@ uint32_t make_idesc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-int do_score_tc(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
+int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
   const Shape& s = c->s;
   const int heads = s.Bt * s.Hkv;
   CUtensorMap qm, km;
@@ -192,39 +187,6 @@ int do_score_tc(dkv_ctx* c, int layer, const void* q, const void* k, float* scor
     tc::score_tc_kernel<tc::kEmit><<<c->tc_emit_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, p, c->tc_stats_grid);
     DKV_LAUNCHED(c);
   }
-  c->scored[layer] = 1;
-  c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
-  return DKV_OK;
-}
-
-int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
-  if (!c->use_simt) return do_score_tc(c, layer, q, k, scores_out, st);
-  const Shape& s = c->s;
-  const uint16_t* qp = static_cast<const uint16_t*>(q);
-  const uint16_t* kp = static_cast<const uint16_t*>(k);
-  const dim3 g1(c->n_split, s.Bt * s.Hkv), g2(c->emit_ctas, s.Bt * s.Hkv);
-  const int threads = c->m_stride;
-  {
-    ProfScope ps(c, DKV_STEP_SCORE_STATS, 1, st);
-    if (s.D == 128)
-      score_stats_simt<128><<<g1, threads, 0, st>>>(qp, kp, c->d_stats, s, c->keys_per_split, c->n_split, c->m_stride);
-    else
-      score_stats_simt<64><<<g1, threads, 0, st>>>(qp, kp, c->d_stats, s, c->keys_per_split, c->n_split, c->m_stride);
-    DKV_LAUNCHED(c);
-  }
-  {
-    ProfScope ps(c, DKV_STEP_SCORE_EMIT, 1, st);
-    if (s.D == 128)
-      score_emit_simt<128><<<g2, threads, 0, st>>>(qp, kp, c->d_stats, c->d_raw, s, c->keys_per_emit, c->n_split, c->m_stride);
-    else
-      score_emit_simt<64><<<g2, threads, 0, st>>>(qp, kp, c->d_stats, c->d_raw, s, c->keys_per_emit, c->n_split, c->m_stride);
-    DKV_LAUNCHED(c);
-  }
-  const size_t total = layer_scores(s);
-  ProfScope ps(c, DKV_STEP_POOL, 1, st);
-  maxpool_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(c->d_raw, c->d_scores + (size_t)layer * total, scores_out,
-                                                                  s.P, s.pool / 2, total);
-  DKV_LAUNCHED(c);
   c->scored[layer] = 1;
   c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
   return DKV_OK;
@@ -341,8 +303,8 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
 }
 
 void free_all(dkv_ctx* c) {
-  cudaFree(c->d_scores); cudaFree(c->d_raw); cudaFree(c->d_idx); cudaFree(c->d_rank); cudaFree(c->d_count);
-  cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_stats); cudaFree(c->d_rb_state); cudaFree(c->d_rb_hist);
+  cudaFree(c->d_scores); cudaFree(c->d_idx); cudaFree(c->d_rank); cudaFree(c->d_count);
+  cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_rb_state); cudaFree(c->d_rb_hist);
   cudaFree(c->d_cnt_gt); cudaFree(c->d_cnt_eq); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
   if (c->prof_recs) {
     for (ProfRec& r : *c->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -413,23 +375,12 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   s.S = cfg->seq_len; s.ws = cfg->window; s.pool = cfg->pool_kernel; s.N = cfg->avg_budget; s.Bl = cfg->layer_max;
   s.m = cfg->update_interval;
   s.G = s.Hq / s.Hkv; s.P = s.S - s.ws; s.M = s.ws * s.G; s.Blc = s.Bl < s.P ? s.Bl : s.P; s.rows = s.Blc + s.ws;
-  c->m_stride = (s.M + 31) / 32 * 32;
   const int heads = s.Bt * s.Hkv;
-  int split = (4 * 148 + heads - 1) / heads;
-  if (split > 64) split = 64;
-  int kps = ((s.S + split - 1) / split + kSimtTileKeys - 1) / kSimtTileKeys * kSimtTileKeys;
-  c->keys_per_split = kps;
-  c->n_split = (s.S + kps - 1) / kps;
-  int kpe = ((s.P + split - 1) / split + kSimtTileKeys - 1) / kSimtTileKeys * kSimtTileKeys;
-  c->keys_per_emit = kpe;
-  c->emit_ctas = (s.P + kpe - 1) / kpe;
   c->sort_n = 2;
   while (c->sort_n < s.Blc) c->sort_n <<= 1;
 
   cudaError_t e = cudaGetDevice(&c->device);
   {
-    const char* impl = getenv("DKV_SCORE_IMPL");
-    c->use_simt = impl && strcmp(impl, "simt") == 0;
     int sms = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
     c->n_sms = sms > 0 ? sms : 1;
@@ -449,13 +400,11 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   const size_t bl = (size_t)s.Bt * s.L;
 #define TRY(call) if (e == cudaSuccess) e = (call)
   TRY(cudaMalloc(&c->d_scores, sizeof(float) * s.L * layer_scores(s)));
-  TRY(cudaMalloc(&c->d_raw, sizeof(float) * layer_scores(s)));
   TRY(cudaMalloc(&c->d_idx, sizeof(int) * s.L * layer_idx(s)));
   TRY(cudaMalloc(&c->d_rank, sizeof(int) * s.L * layer_idx(s)));
   TRY(cudaMalloc(&c->d_count, sizeof(int) * bl));
   TRY(cudaMalloc(&c->d_held, sizeof(int) * bl));
   TRY(cudaMalloc(&c->d_dbg, sizeof(int) * 3 * bl));
-  TRY(cudaMalloc(&c->d_stats, sizeof(float2) * heads * c->n_split * c->m_stride));
   TRY(cudaMalloc(&c->d_rb_state, sizeof(RbState) * s.Bt));
   TRY(cudaMalloc(&c->d_rb_hist, sizeof(unsigned int) * 3 * s.Bt * kRbBins));
   TRY(cudaMalloc(&c->d_cnt_gt, sizeof(unsigned int) * bl));
