@@ -39,6 +39,7 @@ extern "C" {
 #define DKV_ERR_TIMEOUT       -4   /* a bounded device-side wait ran out                           */
 #define DKV_ERR_UNSUPPORTED   -5   /* shape outside the compiled set                               */
 #define DKV_ERR_NOMEM         -6   /* device or host allocation failed                             */
+#define DKV_ERR_TOO_LARGE     -7   /* dkv_score_static: the problem does not fit the static scratch */
 
 #define DKV_MAX_LAYERS        128
 #define DKV_MAX_LAYER_BUDGET  16384  /* Bl  */
@@ -81,6 +82,35 @@ int dkv_reset(dkv_ctx* ctx, void* stream);
  *     scores_out : fp32 [Bt, Hkv, P] optional copy of the result (NULL = keep it in the context only)
  *     bf16 inputs, fp32 accumulation.  Stores the scores as layer `layer` of the context's history. */
 int dkv_score(dkv_ctx* ctx, int32_t layer, const void* q_win, const void* k, float* scores_out, void* stream);
+
+/* Scoring for callers that cannot allocate device memory.  (The paper has no counterpart: this is a
+ * packaging of step (1) above, not a step of the method.)
+ *
+ * Who needs it: programs that must not reach cudaMalloc on this path.  Typical cases are an inference
+ * server that has handed all of the GPU's memory to its own pool, so that a library-side cudaMalloc
+ * would simply fail, and a request path on which cudaMalloc's device-wide synchronisation would stall
+ * every other stream.  dkv_create allocates (history, indices, workspaces), so such callers cannot own
+ * a context; this call needs none.  It calls neither cudaMalloc nor cudaFree nor any allocating
+ * library routine.
+ *
+ * What it does: exactly dkv_score's computation for one layer, same kernels, writing the pooled
+ * scores fp32 [Bt, Hkv, P] to scores_out (required).  Only the scoring fields of cfg are used
+ * (heads, head_dim, batch, seq_len, window, pool_kernel); the whole cfg must still be valid.
+ * Its scratch (partial softmax statistics of sweep 1, plus status words) is a fixed array of
+ * DKV_STATIC_SCRATCH_BYTES inside the library image: every GPU that loads libdkv holds those bytes
+ * until the process exits.  A problem that needs more returns DKV_ERR_TOO_LARGE and launches nothing;
+ * the need is 256 + Bt*Hkv * slots * 2048 bytes with slots about (SM count)/(Bt*Hkv) + 2, i.e. some
+ * 0.3 MB for 8 heads and 2 MB for 512 heads on a 148-SM part.
+ *
+ * The first call on each device looks up the array's device address and sets the kernels' shared
+ * memory attribute (host-side, once).  Make that first call before starting any stream capture.
+ * All calls on a device share the one array, and it keeps whatever the last call left: the call
+ * clears the status words it needs zeroed and overwrites every statistic before reading it, so
+ * calls that follow one another on a stream are independent.  Calls that can overlap on the GPU
+ * (different streams, different host threads) race on the array: serialise them.
+ * q_win : bf16 [Bt, Hq, ws, D];  k : bf16 [Bt, Hkv, S, D];  device pointers, 16-byte aligned. */
+#define DKV_STATIC_SCRATCH_BYTES (4u << 20)
+int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, float* scores_out, void* stream);
 
 /* Store caller-computed scores fp32 [Bt, Hkv, P] (finite, >= 0) as layer `layer` of the history,
  * in place of dkv_score (e.g. scores emitted by a fused prefill attention kernel). */

@@ -14,14 +14,14 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libdkv.so")
 
 EXPORTS = [
-    "dkv_create", "dkv_destroy", "dkv_reset", "dkv_score", "dkv_set_scores", "dkv_select_topk", "dkv_rebudget",
+    "dkv_create", "dkv_destroy", "dkv_reset", "dkv_score", "dkv_score_static", "dkv_set_scores", "dkv_select_topk", "dkv_rebudget",
     "dkv_compact", "dkv_compact_all", "dkv_run_prefill_pass", "dkv_run_prefill_pass_host", "dkv_get_counts",
     "dkv_layer_views", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status", "dkv_profile", "dkv_profile_read", "dkv_launch_count", "dkv_last_cuda_error",
     "dkv_strerror", "dkv_version",
 ]
 
 DKV_OK, DKV_ERR_INVALID_ARG, DKV_ERR_STATE, DKV_ERR_CUDA = 0, -1, -2, -3
-DKV_ERR_TIMEOUT, DKV_ERR_UNSUPPORTED, DKV_ERR_NOMEM = -4, -5, -6
+DKV_ERR_TIMEOUT, DKV_ERR_UNSUPPORTED, DKV_ERR_NOMEM, DKV_ERR_TOO_LARGE = -4, -5, -6, -7
 
 
 class DkvConfig(ctypes.Structure):
@@ -54,6 +54,7 @@ def load() -> ctypes.CDLL:
         "dkv_destroy": [vp],
         "dkv_reset": [vp, vp],
         "dkv_score": [vp, i32, vp, vp, vp, vp],
+        "dkv_score_static": [ctypes.POINTER(DkvConfig), vp, vp, vp, vp],
         "dkv_set_scores": [vp, i32, vp, vp],
         "dkv_select_topk": [vp, i32, vp, vp, vp],
         "dkv_rebudget": [vp, i32, vp, vp],
@@ -151,6 +152,12 @@ def dkv_reset(ctx: int, stream=None) -> None:
 
 def dkv_score(ctx: int, layer: int, q_win, k, scores_out=None, stream=None) -> None:
     _check(load().dkv_score(ctx, layer, _ptr(q_win), _ptr(k), _ptr(scores_out), _stream(stream)), "dkv_score")
+
+
+def dkv_score_static(cfg: DkvConfig, q_win, k, scores_out, stream=None) -> None:
+    """Score one layer without a context and without any device allocation (see include/dkv.h)."""
+    _check(load().dkv_score_static(ctypes.byref(cfg), _ptr(q_win), _ptr(k), _ptr(scores_out), _stream(stream)),
+           "dkv_score_static")
 
 
 def dkv_set_scores(ctx: int, layer: int, scores, stream=None) -> None:

@@ -4,6 +4,7 @@
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -355,6 +356,7 @@ const char* dkv_strerror(int code) {
     case DKV_ERR_TIMEOUT: return "device-side wait timed out";
     case DKV_ERR_UNSUPPORTED: return "shape not supported";
     case DKV_ERR_NOMEM: return "out of memory";
+    case DKV_ERR_TOO_LARGE: return "problem needs more scratch than the static array holds";
     default: return "unknown error";
   }
 }
@@ -583,6 +585,81 @@ int dkv_budget_views(dkv_ctx* c, const int32_t** cnt, const int32_t** z, const i
   if (z) *z = c->d_dbg + bl;
   if (zp) *zp = c->d_dbg + 2 * bl;
   if (held) *held = c->d_held;
+  return DKV_OK;
+}
+
+// ---- scoring for callers that cannot allocate ------------------------------------------------------
+// Scratch of dkv_score_static: [0, 256) status words, then the partial softmax statistics of
+// sweep 1.  The array lives in every GPU that loads the library, from load to exit.  In host code
+// its name is only a handle: the device address comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[DKV_STATIC_SCRATCH_BYTES];
+
+namespace {
+struct StaticSetup { bool done; unsigned char* ptr; int sms; };
+StaticSetup g_static_setup[64];
+std::mutex g_static_mutex;
+}  // namespace
+
+int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, float* scores_out, void* stream) {
+  int rc = validate(cfg);
+  if (rc) return rc;
+  if (!q_win || !k || !scores_out || !aligned16(q_win) || !aligned16(k) || !aligned16(scores_out))
+    return DKV_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DKV_ERR_CUDA;
+  StaticSetup su;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticSetup& g = g_static_setup[dev];
+    if (!g.done) {                           // first call on this device
+      void* ptr = nullptr;
+      if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return DKV_ERR_CUDA;
+      int sms = 0;
+      if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return DKV_ERR_CUDA;
+      if (cudaFuncSetAttribute(tc::score_tc_kernel<tc::kStats>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               tc::kSmemBytes) != cudaSuccess ||
+          cudaFuncSetAttribute(tc::score_tc_kernel<tc::kEmit>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               tc::kSmemBytes) != cudaSuccess)
+        return DKV_ERR_CUDA;
+      g.ptr = static_cast<unsigned char*>(ptr);
+      g.sms = sms;
+      g.done = true;
+    }
+    su = g;
+  }
+  const int G = cfg->n_q_heads / cfg->n_kv_heads, heads = cfg->batch * cfg->n_kv_heads;
+  const int S = cfg->seq_len, P = S - cfg->window, M = cfg->window * G, D = cfg->head_dim;
+  const int tph = (S + tc::kTileKeys - 1) / tc::kTileKeys;
+  const long long total_tiles = (long long)heads * tph;
+  const int stats_grid = (int)(total_tiles < su.sms ? total_tiles : su.sms);
+  const long long out_tiles = ((long long)heads * P + tc::kTileKeys - 1) / tc::kTileKeys;
+  const int emit_grid = (int)(out_tiles < su.sms ? out_tiles : su.sms);
+  int slots = 1;
+  for (int bh = 0; bh < heads; ++bh) {
+    const int lo = tc::tile_owner((long long)bh * tph, total_tiles, stats_grid);
+    const int hi = tc::tile_owner((long long)(bh + 1) * tph - 1, total_tiles, stats_grid);
+    if (hi - lo + 1 > slots) slots = hi - lo + 1;
+  }
+  const unsigned long long need = 256ull + (unsigned long long)heads * slots * 256ull * sizeof(float2);
+  if (need > DKV_STATIC_SCRATCH_BYTES) return DKV_ERR_TOO_LARGE;
+  cudaStream_t st = as_stream(stream);
+  CUtensorMap qm, km;
+  if (!make_map(&qm, q_win, D, M, heads) || !make_map(&km, k, D, S, heads)) return DKV_ERR_CUDA;
+  if (cudaMemsetAsync(su.ptr, 0, 256, st) != cudaSuccess) return DKV_ERR_CUDA;   // status words start at zero
+  tc::Params p;
+  p.S = S; p.P = P; p.ws = cfg->window; p.M = M; p.D = D; p.heads = heads; p.half = cfg->pool_kernel / 2;
+  p.tph = tph; p.nq16 = (M + 15) / 16 * 16; p.nmblk = (M + 127) / 128;
+  p.slots = slots; p.m_stride = 256;
+  p.scale2 = kLog2e / sqrtf((float)D);
+  p.stats = reinterpret_cast<float2*>(su.ptr + 256);
+  p.scores = scores_out; p.copy_out = nullptr;
+  p.status = reinterpret_cast<int*>(su.ptr);
+  p.idesc = make_idesc(128, 128);
+  tc::score_tc_kernel<tc::kStats><<<stats_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, p, stats_grid);
+  if (cudaPeekAtLastError() != cudaSuccess) return DKV_ERR_CUDA;
+  p.idesc = make_idesc(128, p.nq16);
+  tc::score_tc_kernel<tc::kEmit><<<emit_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, p, stats_grid);
+  if (cudaPeekAtLastError() != cudaSuccess) return DKV_ERR_CUDA;
   return DKV_OK;
 }
 
