@@ -300,11 +300,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="dkv", choices=["dkv", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers of the workload")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
+    if args.layers:
+        w = w.with_(name=f"{w.name}[:{args.layers}]", L=args.layers)
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) != 0:
             return 0
