@@ -37,8 +37,10 @@ struct dkv_ctx {
   int* d_status;        // [8]
   int sort_n;
   // tensor-core scoring
-  int n_sms, tc_stats_grid, tc_emit_grid, tc_slots;
-  float2* d_tc_stats;   // [Bt*Hkv][tc_slots][256]
+  int n_sms, tc_grid, tc_slots;
+  float2* d_tc_stats;   // [3][Bt*Hkv][tc_slots][256]: partial softmax statistics, three layers in rotation
+  cudaStream_t side;    // second stream of dkv_run_prefill_pass (select / gather / rebudget / shrink)
+  cudaEvent_t ev_fork, ev_join, ev_scored[DKV_MAX_LAYERS];
   // host state
   uint8_t scored[DKV_MAX_LAYERS], selected[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
   long long launches;
@@ -160,34 +162,49 @@ uint32_t make_idesc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
+// Parameters of one sweep over one layer; `buf` picks the statistics scratch (layers alternate).
+bool make_job(dkv_ctx* c, int mode, int layer, const void* q, const void* k, float* scores_out, int buf,
+              CUtensorMap* qm, CUtensorMap* km, tc::Params* p) {
   const Shape& s = c->s;
   const int heads = s.Bt * s.Hkv;
-  CUtensorMap qm, km;
-  if (!make_map(&qm, q, s.D, s.M, heads) || !make_map(&km, k, s.D, s.S, heads)) return DKV_ERR_CUDA;
-  tc::Params p;
-  p.S = s.S; p.P = s.P; p.ws = s.ws; p.M = s.M; p.D = s.D; p.heads = heads; p.half = s.pool / 2;
-  p.tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
-  p.nq16 = (s.M + 15) / 16 * 16;
-  p.nmblk = (s.M + 127) / 128;
-  p.slots = c->tc_slots; p.m_stride = 256;
-  p.scale2 = kLog2e / sqrtf((float)s.D);
-  p.stats = c->d_tc_stats;
-  p.scores = c->d_scores + (size_t)layer * layer_scores(s);
-  p.copy_out = scores_out;
-  p.status = c->d_status;
-  {
-    ProfScope ps(c, DKV_STEP_SCORE_STATS, 1, st);
-    p.idesc = make_idesc(128, 128);
-    tc::score_tc_kernel<tc::kStats><<<c->tc_stats_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, p, c->tc_stats_grid);
-    DKV_LAUNCHED(c);
-  }
-  {
-    ProfScope ps(c, DKV_STEP_SCORE_EMIT, 1, st);
-    p.idesc = make_idesc(128, p.nq16);
-    tc::score_tc_kernel<tc::kEmit><<<c->tc_emit_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, p, c->tc_stats_grid);
-    DKV_LAUNCHED(c);
-  }
+  if (!make_map(qm, q, s.D, s.M, heads) || !make_map(km, k, s.D, s.S, heads)) return false;
+  p->S = s.S; p->P = s.P; p->ws = s.ws; p->M = s.M; p->D = s.D; p->heads = heads; p->half = s.pool / 2;
+  p->tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
+  p->nq16 = (s.M + 15) / 16 * 16;
+  p->nmblk = (s.M + 127) / 128;
+  p->slots = c->tc_slots; p->m_stride = 256;
+  p->scale2 = kLog2e / sqrtf((float)s.D);
+  p->stats = c->d_tc_stats + (size_t)buf * heads * c->tc_slots * 256;
+  p->scores = c->d_scores + (size_t)layer * layer_scores(s);
+  p->copy_out = scores_out;
+  p->status = c->d_status;
+  p->stats_grid = c->tc_grid;
+  p->mode = mode;
+  p->idesc = mode == tc::kStats ? make_idesc(128, 128) : make_idesc(128, p->nq16);
+  return true;
+}
+
+// One launch: sweep 1 of `stats_layer` (if >= 0), then sweep 2 of `emit_layer` (if >= 0).
+int launch_score(dkv_ctx* c, int stats_layer, const void* sq, const void* sk, int emit_layer, const void* eq,
+                 const void* ek, float* scores_out, cudaStream_t st) {
+  CUtensorMap qm0, km0, qm1, km1;
+  tc::Params j0, j1;
+  memset(&j0, 0, sizeof j0); memset(&j1, 0, sizeof j1);
+  j0.mode = j1.mode = tc::kNone;
+  if (stats_layer >= 0 && !make_job(c, tc::kStats, stats_layer, sq, sk, nullptr, stats_layer % 3, &qm0, &km0, &j0)) return DKV_ERR_CUDA;
+  if (emit_layer >= 0 && !make_job(c, tc::kEmit, emit_layer, eq, ek, scores_out, emit_layer % 3, &qm1, &km1, &j1)) return DKV_ERR_CUDA;
+  if (stats_layer < 0) { qm0 = qm1; km0 = km1; }
+  if (emit_layer < 0) { qm1 = qm0; km1 = km0; }
+  ProfScope ps(c, stats_layer >= 0 ? DKV_STEP_SCORE_STATS : DKV_STEP_SCORE_EMIT, 1, st);
+  tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm0, km0, qm1, km1, j0, j1);
+  DKV_LAUNCHED(c);
+  return DKV_OK;
+}
+
+int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
+  int rc = launch_score(c, layer, q, k, -1, nullptr, nullptr, nullptr, st);
+  if (rc) return rc;
+  if ((rc = launch_score(c, -1, nullptr, nullptr, layer, q, k, scores_out, st))) return rc;
   c->scored[layer] = 1;
   c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
   return DKV_OK;
@@ -285,21 +302,37 @@ int do_reset(dkv_ctx* c, cudaStream_t st) {
   return DKV_OK;
 }
 
+// Algorithm 1's loop.  The scoring launches run back to back on `st` (launch l = sweep 1 of layer l
+// followed by sweep 2 of layer l-1); everything that consumes a layer's scores (select, gather, and
+// every m layers rebudget + shrink) runs on the context's second stream behind an event, so that it
+// overlaps the scoring of the following layers.  `st` rejoins the second stream at the end.
 int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* const* v, void* const* kb,
             void* const* vb, cudaStream_t st) {
   const Shape& s = c->s;
   int rc = do_reset(c, st);
   if (rc) return rc;
-  for (int l = 0; l < s.L; ++l) {
-    if ((rc = do_score(c, l, q[l], k[l], nullptr, st))) return rc;
-    if ((rc = do_select(c, l, nullptr, nullptr, st))) return rc;
-    if ((rc = do_gather(c, l, k[l], v[l], kb[l], vb[l], st))) return rc;
-    const bool update = ((l + 1) % s.m == 0) || (l + 1 == s.L && s.L % s.m != 0);
+  cudaStream_t sd = c->side;
+  DKV_CUDA(c, cudaEventRecord(c->ev_fork, st));
+  DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_fork, 0));
+  for (int l = 0; l <= s.L; ++l) {
+    const int sl = l < s.L ? l : -1, el = l - 1;
+    if ((rc = launch_score(c, sl, sl >= 0 ? q[sl] : nullptr, sl >= 0 ? k[sl] : nullptr, el, el >= 0 ? q[el] : nullptr,
+                           el >= 0 ? k[el] : nullptr, nullptr, st)))
+      return rc;
+    if (el < 0) continue;
+    c->scored[el] = 1;
+    DKV_CUDA(c, cudaEventRecord(c->ev_scored[el], st));
+    DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_scored[el], 0));
+    if ((rc = do_select(c, el, nullptr, nullptr, sd))) return rc;
+    if ((rc = do_gather(c, el, k[el], v[el], kb[el], vb[el], sd))) return rc;
+    const bool update = ((el + 1) % s.m == 0) || (el + 1 == s.L && s.L % s.m != 0);
     if (update) {
-      if ((rc = do_rebudget(c, l + 1, nullptr, st))) return rc;
-      if ((rc = do_shrink(c, 0, l + 1, kb, vb, st))) return rc;
+      if ((rc = do_rebudget(c, el + 1, nullptr, sd))) return rc;
+      if ((rc = do_shrink(c, 0, el + 1, kb, vb, sd))) return rc;
     }
   }
+  DKV_CUDA(c, cudaEventRecord(c->ev_join, sd));
+  DKV_CUDA(c, cudaStreamWaitEvent(st, c->ev_join, 0));
   return DKV_OK;
 }
 
@@ -307,6 +340,10 @@ void free_all(dkv_ctx* c) {
   cudaFree(c->d_scores); cudaFree(c->d_idx); cudaFree(c->d_rank); cudaFree(c->d_count);
   cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_rb_state); cudaFree(c->d_rb_hist);
   cudaFree(c->d_cnt_gt); cudaFree(c->d_cnt_eq); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
+  if (c->side) cudaStreamDestroy(c->side);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
+  for (int l = 0; l < DKV_MAX_LAYERS; ++l) if (c->ev_scored[l]) cudaEventDestroy(c->ev_scored[l]);
   if (c->prof_recs) {
     for (ProfRec& r : *c->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     delete c->prof_recs;
@@ -388,13 +425,11 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
     c->n_sms = sms > 0 ? sms : 1;
     const int tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
     const long long total_tiles = (long long)heads * tph;
-    c->tc_stats_grid = (int)(total_tiles < c->n_sms ? total_tiles : c->n_sms);
-    const long long out_tiles = ((long long)heads * s.P + tc::kTileKeys - 1) / tc::kTileKeys;
-    c->tc_emit_grid = (int)(out_tiles < c->n_sms ? out_tiles : c->n_sms);
+    c->tc_grid = (int)(total_tiles < c->n_sms ? total_tiles : c->n_sms);
     int slots = 1;
     for (int bh = 0; bh < heads; ++bh) {
-      const int lo = tc::tile_owner((long long)bh * tph, total_tiles, c->tc_stats_grid);
-      const int hi = tc::tile_owner((long long)(bh + 1) * tph - 1, total_tiles, c->tc_stats_grid);
+      const int lo = tc::tile_owner((long long)bh * tph, total_tiles, c->tc_grid);
+      const int hi = tc::tile_owner((long long)(bh + 1) * tph - 1, total_tiles, c->tc_grid);
       if (hi - lo + 1 > slots) slots = hi - lo + 1;
     }
     c->tc_slots = slots;
@@ -411,9 +446,12 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMalloc(&c->d_rb_hist, sizeof(unsigned int) * 3 * s.Bt * kRbBins));
   TRY(cudaMalloc(&c->d_cnt_gt, sizeof(unsigned int) * bl));
   TRY(cudaMalloc(&c->d_cnt_eq, sizeof(unsigned int) * bl));
-  TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * heads * c->tc_slots * 256));
-  TRY(cudaFuncSetAttribute(tc::score_tc_kernel<tc::kStats>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
-  TRY(cudaFuncSetAttribute(tc::score_tc_kernel<tc::kEmit>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * 3 * heads * c->tc_slots * 256));
+  TRY(cudaFuncSetAttribute(tc::score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  TRY(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
+  TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
+  TRY(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
+  for (int l = 0; l < s.L; ++l) TRY(cudaEventCreateWithFlags(&c->ev_scored[l], cudaEventDisableTiming));
   TRY(cudaMalloc(&c->d_status, sizeof(int) * 8));
   TRY(cudaMemset(c->d_status, 0, sizeof(int) * 8));
   TRY(cudaMemset(c->d_count, 0, sizeof(int) * bl));
@@ -616,10 +654,8 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
       if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return DKV_ERR_CUDA;
       int sms = 0;
       if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return DKV_ERR_CUDA;
-      if (cudaFuncSetAttribute(tc::score_tc_kernel<tc::kStats>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               tc::kSmemBytes) != cudaSuccess ||
-          cudaFuncSetAttribute(tc::score_tc_kernel<tc::kEmit>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               tc::kSmemBytes) != cudaSuccess)
+      if (cudaFuncSetAttribute(tc::score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes) !=
+          cudaSuccess)
         return DKV_ERR_CUDA;
       g.ptr = static_cast<unsigned char*>(ptr);
       g.sms = sms;
@@ -631,13 +667,11 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   const int S = cfg->seq_len, P = S - cfg->window, M = cfg->window * G, D = cfg->head_dim;
   const int tph = (S + tc::kTileKeys - 1) / tc::kTileKeys;
   const long long total_tiles = (long long)heads * tph;
-  const int stats_grid = (int)(total_tiles < su.sms ? total_tiles : su.sms);
-  const long long out_tiles = ((long long)heads * P + tc::kTileKeys - 1) / tc::kTileKeys;
-  const int emit_grid = (int)(out_tiles < su.sms ? out_tiles : su.sms);
+  const int grid = (int)(total_tiles < su.sms ? total_tiles : su.sms);
   int slots = 1;
   for (int bh = 0; bh < heads; ++bh) {
-    const int lo = tc::tile_owner((long long)bh * tph, total_tiles, stats_grid);
-    const int hi = tc::tile_owner((long long)(bh + 1) * tph - 1, total_tiles, stats_grid);
+    const int lo = tc::tile_owner((long long)bh * tph, total_tiles, grid);
+    const int hi = tc::tile_owner((long long)(bh + 1) * tph - 1, total_tiles, grid);
     if (hi - lo + 1 > slots) slots = hi - lo + 1;
   }
   const unsigned long long need = 256ull + (unsigned long long)heads * slots * 256ull * sizeof(float2);
@@ -646,7 +680,9 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   CUtensorMap qm, km;
   if (!make_map(&qm, q_win, D, M, heads) || !make_map(&km, k, D, S, heads)) return DKV_ERR_CUDA;
   if (cudaMemsetAsync(su.ptr, 0, 256, st) != cudaSuccess) return DKV_ERR_CUDA;   // status words start at zero
-  tc::Params p;
+  tc::Params p, none;
+  memset(&none, 0, sizeof none);
+  none.mode = tc::kNone;
   p.S = S; p.P = P; p.ws = cfg->window; p.M = M; p.D = D; p.heads = heads; p.half = cfg->pool_kernel / 2;
   p.tph = tph; p.nq16 = (M + 15) / 16 * 16; p.nmblk = (M + 127) / 128;
   p.slots = slots; p.m_stride = 256;
@@ -654,11 +690,14 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   p.stats = reinterpret_cast<float2*>(su.ptr + 256);
   p.scores = scores_out; p.copy_out = nullptr;
   p.status = reinterpret_cast<int*>(su.ptr);
+  p.stats_grid = grid;
+  p.mode = tc::kStats;
   p.idesc = make_idesc(128, 128);
-  tc::score_tc_kernel<tc::kStats><<<stats_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, p, stats_grid);
+  tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, qm, km, p, none);
   if (cudaPeekAtLastError() != cudaSuccess) return DKV_ERR_CUDA;
+  p.mode = tc::kEmit;
   p.idesc = make_idesc(128, p.nq16);
-  tc::score_tc_kernel<tc::kEmit><<<emit_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, p, stats_grid);
+  tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, qm, km, none, p);
   if (cudaPeekAtLastError() != cudaSuccess) return DKV_ERR_CUDA;
   return DKV_OK;
 }

@@ -9,9 +9,12 @@
 //                     with no cross-thread reduction; the CTA then max-pools its key range.
 // Both sweeps share one pipeline: a TMA producer warp streams 128-key tiles of K (bf16, 128-byte
 // swizzle) through a shared-memory ring, one thread issues tcgen05.mma into double-buffered TMEM
-// accumulators, and two groups of four warps read the accumulators back with tcgen05.ld.
+// accumulators, and sixteen warps read the accumulators back with tcgen05.ld (four warps per TMEM
+// lane quadrant, each taking a quarter of the columns).
 // Work is split evenly: the flattened (head, key tile) space for sweep 1 and the flattened
 // (head, prefix position) space for sweep 2 are cut into one contiguous slice per CTA.
+// One launch runs up to two jobs back to back through the same pipeline (sweep 1 of one layer, then
+// sweep 2 of the layer before it), so the fixed cost of a launch is paid once per layer.
 #pragma once
 #include <cuda.h>
 #include "common.cuh"
@@ -21,17 +24,20 @@ namespace tc {
 
 constexpr int kTileKeys = 128;
 constexpr int kStages = 4;                 // K tiles in flight
-constexpr int kThreads = 320;              // warp 0: TMA, warp 1: MMA, warps 2..9: two softmax groups
-constexpr int kSoftmaxThreads = 256;
-constexpr int kMaxSegTiles = 16;           // sweep 2: tiles per pooled segment
+constexpr int kThreads = 576;              // warp 0: TMA, warp 1: MMA, warps 2..17: softmax
+constexpr int kSoftmaxThreads = 512;
+constexpr int kParts = 4;                  // softmax warps per TMEM lane quadrant
+constexpr int kMaxSegTiles = 8;            // sweep 2: tiles per pooled segment
+constexpr int kStageCols = 256;            // TMEM columns per accumulator stage
 constexpr int kHalfBytes = 128 * 128;      // one 128-row x 64-column bf16 box
 constexpr int kQRegion = 2 * 2 * kHalfBytes;          // up to 256 rows x 128 columns
 constexpr int kKRegion = kStages * 2 * kHalfBytes;    // ring of 128 x 128 tiles
-constexpr int kSmemBytes = 1024 /*align*/ + kQRegion + kKRegion + 4096 /*lse, merge*/ +
-                           kMaxSegTiles * kTileKeys * 4 /*raw*/ + 256 /*barriers*/;
+constexpr int kMiscBytes = 1024 /*lse*/ + 3 * 256 * 8 /*merge*/;
+constexpr int kRawBytes = kParts * kMaxSegTiles * kTileKeys * 4;
+constexpr int kSmemBytes = 1024 /*align*/ + kQRegion + kKRegion + kMiscBytes + kRawBytes + 256 /*barriers*/;
 constexpr long long kWaitCycles = 4000000000ll;       // ~2 s: a wait that long is reported, not spun on
 
-enum Mode { kStats = 0, kEmit = 1 };
+enum Mode { kNone = 0, kStats = 1, kEmit = 2 };
 
 struct Params {
   int S, P, ws, M, D, heads, half;
@@ -46,6 +52,8 @@ struct Params {
   float* scores;           // [heads][P] pooled scores (sweep 2)
   float* copy_out;         // optional second copy
   int* status;             // device status words; [0] = first error
+  int stats_grid;          // CTAs of the launch that ran sweep 1 for this layer
+  int mode;                // kNone: nothing to do
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -110,6 +118,24 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory operand descriptor: K-major, 128-byte swizzle, rows 128 B apart, 8-row groups 1024 B apart.
@@ -132,12 +158,12 @@ struct Seg {
   bool new_head;
 };
 
-template <int MODE>
 struct SegIter {
   long long u, u_end;
-  int uph, half, cur_bh;
+  int uph, half, cur_bh, mode;
   __device__ SegIter(const Params& p, int cta, int grid) {
-    uph = MODE == kStats ? p.tph : p.P;
+    mode = p.mode;
+    uph = mode == kStats ? p.tph : p.P;
     const long long total = (long long)p.heads * uph;
     u = total * cta / grid;
     u_end = total * (cta + 1) / grid;
@@ -149,10 +175,10 @@ struct SegIter {
     const int bh = (int)(u / uph), off = (int)(u % uph);
     long long e = (long long)(bh + 1) * uph;
     if (e > u_end) e = u_end;
-    if (MODE == kEmit && e > u + (kMaxSegTiles * kTileKeys - 2 * half)) e = u + (kMaxSegTiles * kTileKeys - 2 * half);
+    if (mode == kEmit && e > u + (kMaxSegTiles * kTileKeys - 2 * half)) e = u + (kMaxSegTiles * kTileKeys - 2 * half);
     const int len = (int)(e - u);
     s.bh = bh;
-    if (MODE == kStats) {
+    if (mode == kStats) {
       s.key0 = off * kTileKeys; s.ntiles = len; s.out0 = s.out1 = 0;
     } else {
       s.out0 = off; s.out1 = off + len; s.key0 = off - half;
@@ -171,18 +197,19 @@ __host__ __device__ __forceinline__ int tile_owner(long long x, long long total,
 }
 
 // ------------------------------------------------------------------------------------------ kernel
-template <int MODE>
+// job0 uses (q_map0, k_map0), job1 uses (q_map1, k_map1); a job with mode kNone is skipped.
 __global__ void __launch_bounds__(kThreads, 1)
-score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map, const Params p,
-                int stats_grid) {
+score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constant__ CUtensorMap k_map0,
+                const __grid_constant__ CUtensorMap q_map1, const __grid_constant__ CUtensorMap k_map1,
+                const __grid_constant__ Params job0, const __grid_constant__ Params job1) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* q_smem = smem;                              // [half][256 rows][128 B]
   uint8_t* k_smem = smem + kQRegion;                   // [stage][half][128 rows][128 B]
   float* lse_s = reinterpret_cast<float*>(k_smem + kKRegion);          // [256] lse2 per window row (sweep 2)
-  float2* merge_s = reinterpret_cast<float2*>(lse_s + 256);            // [256] group-B partials (sweep 1)
-  float* raw_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(lse_s) + 4096);   // [16 * 128]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(raw_s + kMaxSegTiles * kTileKeys);
+  float2* merge_s = reinterpret_cast<float2*>(lse_s + 256);            // [3][256] partials of column parts 1..3 (sweep 1)
+  float* raw_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(lse_s) + kMiscBytes);   // [part][8 * 128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(raw_s) + kRawBytes);
   // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2], q_full
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
@@ -194,14 +221,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   const uint32_t QFULL = bar0 + 8u * (2 * kStages + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int halves = p.D / 64;
-  const uint32_t tile_bytes = (uint32_t)halves * kHalfBytes;
   volatile int* abort_flag = &abort_s;
 
   if (threadIdx.x == 0) {
     abort_s = 0;
     for (int s = 0; s < kStages; ++s) { mbar_init(FULL(s), 1); mbar_init(EMPTY(s), 1); }
-    for (int t = 0; t < 2; ++t) { mbar_init(TFULL(t), 1); mbar_init(TEMPTY(t), 4); }
+    for (int t = 0; t < 2; ++t) { mbar_init(TFULL(t), 1); mbar_init(TEMPTY(t), 16); }
     mbar_init(QFULL, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -213,215 +238,258 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
-  const int stage_cols = MODE == kStats ? p.nmblk * 128 : 256;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      SegIter<MODE> it(p, blockIdx.x, gridDim.x);
-      Seg sg;
-      int tile = 0, nq = 0;
-      while (it.next(sg)) {
-        if (sg.new_head) {
-          if (tile > 0) {   // all MMAs that read the previous head's queries must have finished
-            const int last = tile - 1;
-            mbar_wait(EMPTY(last % kStages), (last / kStages) & 1, abort_flag, p.status, 101);
+      int tile = 0;
+      for (int jb = 0; jb < 2; ++jb) {
+        const Params& p = jb ? job1 : job0;
+        if (p.mode == kNone) continue;
+        const CUtensorMap* q_map = jb ? &q_map1 : &q_map0;
+        const CUtensorMap* k_map = jb ? &k_map1 : &k_map0;
+        const int halves = p.D / 64;
+        const uint32_t tile_bytes = (uint32_t)halves * kHalfBytes;
+        SegIter it(p, blockIdx.x, gridDim.x);
+        Seg sg;
+        while (it.next(sg)) {
+          if (sg.new_head) {
+            if (tile > 0) {   // every MMA that read the previous queries must have finished
+              const int last = tile - 1;
+              mbar_wait(EMPTY(last % kStages), (last / kStages) & 1, abort_flag, p.status, 101);
+            }
+            if (!*abort_flag) {
+              mbar_expect_tx(QFULL, (uint32_t)(p.nmblk * halves) * kHalfBytes);
+              for (int h = 0; h < halves; ++h)
+                for (int mb = 0; mb < p.nmblk; ++mb)
+                  tma_load_3d(smem_u32(q_smem + h * (2 * kHalfBytes) + mb * kHalfBytes), q_map, QFULL, 64 * h, 128 * mb, sg.bh);
+            }
           }
-          if (!*abort_flag) {
-            mbar_expect_tx(QFULL, (uint32_t)(p.nmblk * halves) * kHalfBytes);
+          for (int i = 0; i < sg.ntiles; ++i, ++tile) {
+            const int s = tile % kStages, n = tile / kStages;
+            mbar_wait(EMPTY(s), (n & 1) ^ 1, abort_flag, p.status, 102);
+            if (*abort_flag) break;
+            mbar_expect_tx(FULL(s), tile_bytes);
             for (int h = 0; h < halves; ++h)
-              for (int mb = 0; mb < p.nmblk; ++mb)
-                tma_load_3d(smem_u32(q_smem + h * (2 * kHalfBytes) + mb * kHalfBytes), &q_map, QFULL, 64 * h, 128 * mb, sg.bh);
+              tma_load_3d(smem_u32(k_smem + (s * 2 + h) * kHalfBytes), k_map, FULL(s), 64 * h, sg.key0 + i * kTileKeys, sg.bh);
           }
-          ++nq;
-        }
-        for (int i = 0; i < sg.ntiles; ++i, ++tile) {
-          const int s = tile % kStages, n = tile / kStages;
-          mbar_wait(EMPTY(s), (n & 1) ^ 1, abort_flag, p.status, 102);
           if (*abort_flag) break;
-          mbar_expect_tx(FULL(s), tile_bytes);
-          for (int h = 0; h < halves; ++h)
-            tma_load_3d(smem_u32(k_smem + (s * 2 + h) * kHalfBytes), &k_map, FULL(s), 64 * h, sg.key0 + i * kTileKeys, sg.bh);
         }
-        if (*abort_flag) break;
       }
-      (void)nq;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      SegIter<MODE> it(p, blockIdx.x, gridDim.x);
-      Seg sg;
       int tile = 0, nq = 0;
-      const int ksteps = p.D / 16;
-      while (it.next(sg)) {
-        if (sg.new_head) { mbar_wait(QFULL, nq & 1, abort_flag, p.status, 103); ++nq; }
-        for (int i = 0; i < sg.ntiles; ++i, ++tile) {
-          const int s = tile % kStages, n = tile / kStages, t = tile & 1, nt = tile >> 1;
-          mbar_wait(FULL(s), n & 1, abort_flag, p.status, 104);
-          mbar_wait(TEMPTY(t), (nt & 1) ^ 1, abort_flag, p.status, 105);
-          tc_fence_after();
-          const uint32_t d_tmem = tmem_base + (uint32_t)(t * stage_cols);
-          if (MODE == kStats) {
-            for (int mb = 0; mb < p.nmblk; ++mb)
+      for (int jb = 0; jb < 2; ++jb) {
+        const Params& p = jb ? job1 : job0;
+        if (p.mode == kNone) continue;
+        const int ksteps = p.D / 16;
+        SegIter it(p, blockIdx.x, gridDim.x);
+        Seg sg;
+        while (it.next(sg)) {
+          if (sg.new_head) { mbar_wait(QFULL, nq & 1, abort_flag, p.status, 103); ++nq; }
+          for (int i = 0; i < sg.ntiles; ++i, ++tile) {
+            const int s = tile % kStages, n = tile / kStages, t = tile & 1, nt = tile >> 1;
+            mbar_wait(FULL(s), n & 1, abort_flag, p.status, 104);
+            mbar_wait(TEMPTY(t), (nt & 1) ^ 1, abort_flag, p.status, 105);
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(t * kStageCols);
+            if (p.mode == kStats) {
+              for (int mb = 0; mb < p.nmblk; ++mb)
+                for (int ks = 0; ks < ksteps; ++ks) {
+                  const uint64_t a = smem_desc(smem_u32(q_smem + (ks >> 2) * (2 * kHalfBytes) + mb * kHalfBytes) + (ks & 3) * 32);
+                  const uint64_t b = smem_desc(smem_u32(k_smem + (s * 2 + (ks >> 2)) * kHalfBytes) + (ks & 3) * 32);
+                  tc_mma(d_tmem + mb * 128, a, b, p.idesc, ks > 0);
+                }
+            } else {
               for (int ks = 0; ks < ksteps; ++ks) {
-                const uint64_t a = smem_desc(smem_u32(q_smem + (ks >> 2) * (2 * kHalfBytes) + mb * kHalfBytes) + (ks & 3) * 32);
-                const uint64_t b = smem_desc(smem_u32(k_smem + (s * 2 + (ks >> 2)) * kHalfBytes) + (ks & 3) * 32);
-                tc_mma(d_tmem + mb * 128, a, b, p.idesc, ks > 0);
+                const uint64_t a = smem_desc(smem_u32(k_smem + (s * 2 + (ks >> 2)) * kHalfBytes) + (ks & 3) * 32);
+                const uint64_t b = smem_desc(smem_u32(q_smem + (ks >> 2) * (2 * kHalfBytes)) + (ks & 3) * 32);
+                tc_mma(d_tmem, a, b, p.idesc, ks > 0);
               }
-          } else {
-            for (int ks = 0; ks < ksteps; ++ks) {
-              const uint64_t a = smem_desc(smem_u32(k_smem + (s * 2 + (ks >> 2)) * kHalfBytes) + (ks & 3) * 32);
-              const uint64_t b = smem_desc(smem_u32(q_smem + (ks >> 2) * (2 * kHalfBytes)) + (ks & 3) * 32);
-              tc_mma(d_tmem, a, b, p.idesc, ks > 0);
             }
+            tc_commit(EMPTY(s));      // the K slot may be refilled once these MMAs have read it
+            tc_commit(TFULL(t));      // the accumulator is complete
           }
-          tc_commit(EMPTY(s));      // the K slot may be refilled once these MMAs have read it
-          tc_commit(TFULL(t));      // the accumulator is complete
         }
       }
     }
   } else {
     // ------------------------------------------------------------------ softmax warps
-    const int sw = warp - 2;                   // 0..7
-    const int grp = sw >> 2;                   // group 0 takes even tiles, group 1 odd tiles
+    const int part = (warp - 2) >> 2;          // which quarter of the accumulator columns
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
     const int row = quad * 32 + lane;          // TMEM lane = window row (sweep 1) or key within the tile (sweep 2)
-    const int sid = threadIdx.x - 64;          // 0..255 among the softmax threads
-    SegIter<MODE> it(p, blockIdx.x, gridDim.x);
-    Seg sg;
+    const int sid = threadIdx.x - 64;          // 0..511 among the softmax threads
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     int tile = 0;
-    while (it.next(sg)) {
-      if (MODE == kStats) {
-        float mx[2] = {-INFINITY, -INFINITY}, sum[2] = {0.f, 0.f};
-        int limit[2];
+    for (int jb = 0; jb < 2; ++jb) {
+      const Params& p = jb ? job1 : job0;
+      if (p.mode == kNone) continue;
+      SegIter it(p, blockIdx.x, gridDim.x);
+      Seg sg;
+      while (it.next(sg)) {
+        if (p.mode == kStats) {
+          // ------------------------------------------------------------ sweep 1: (max, sum) per window row
+          float mx[2] = {-INFINITY, -INFINITY}, sum[2] = {0.f, 0.f};
+          const int limit0 = p.P + (row % p.ws), limit1 = p.P + ((row + 128) % p.ws);
+          for (int i = 0; i < sg.ntiles; ++i, ++tile) {
+            const int t = tile & 1, nt = tile >> 1;
+            mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 106);
+            tc_fence_after();
+            const uint32_t taddr = lane_addr + (uint32_t)(t * kStageCols + part * 32);
+            const int kb = sg.key0 + i * kTileKeys + part * 32;
+            const bool need_mask = kb + 31 > p.P;
 #pragma unroll
-        for (int mb = 0; mb < 2; ++mb) limit[mb] = p.P + ((row + 128 * mb) % p.ws);
-        for (int i = 0; i < sg.ntiles; ++i, ++tile) {
-          if ((tile & 1) != grp) continue;
-          const int t = tile & 1, nt = tile >> 1;
-          mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 106);
-          tc_fence_after();
-          const int kb = sg.key0 + i * kTileKeys;
-          const bool need_mask = kb + kTileKeys - 1 > p.P;
-#pragma unroll
-          for (int mb = 0; mb < 2; ++mb) {
-            if (mb >= p.nmblk) break;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * stage_cols + mb * 128);
-#pragma unroll 1
-            for (int c = 0; c < 8; ++c) {
-              float x[16];
-              tc_ld16(taddr + c * 16, x);
+            for (int mb = 0; mb < 2; ++mb) {
+              if (mb >= p.nmblk) break;
+              float xv[32];
+              tc_ld32(taddr + mb * 128, xv);
               tc_wait_ld();
-              if (need_mask) {
-#pragma unroll
-                for (int e = 0; e < 16; ++e) if (kb + c * 16 + e > limit[mb]) x[e] = -INFINITY;
+              if (mb + 1 == p.nmblk) {                         // last read of this stage: release it
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(TEMPTY(t));
               }
-              float cm = x[0];
+              if (need_mask) {
+                const int limit = mb ? limit1 : limit0;
 #pragma unroll
-              for (int e = 1; e < 16; ++e) cm = fmaxf(cm, x[e]);
+                for (int e = 0; e < 32; ++e) if (kb + e > limit) xv[e] = -INFINITY;
+              }
+              float cm = fmax3(xv[0], xv[1], xv[2]);
+#pragma unroll
+              for (int e = 3; e < 31; e += 2) cm = fmax3(cm, xv[e], xv[e + 1]);
+              cm = fmaxf(cm, xv[31]);
               if (cm == -INFINITY) continue;
               const float mnew = fmaxf(mx[mb], cm * p.scale2);
               if (mnew > mx[mb]) { sum[mb] *= fast_exp2(mx[mb] - mnew); mx[mb] = mnew; }
               float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
               const float neg = -mx[mb];
 #pragma unroll
-              for (int e = 0; e < 16; e += 4) {
-                s0 += fast_exp2(fmaf(x[e], p.scale2, neg));
-                s1 += fast_exp2(fmaf(x[e + 1], p.scale2, neg));
-                s2 += fast_exp2(fmaf(x[e + 2], p.scale2, neg));
-                s3 += fast_exp2(fmaf(x[e + 3], p.scale2, neg));
+              for (int e = 0; e < 32; e += 4) {
+                s0 += fast_exp2(fmaf(xv[e], p.scale2, neg));
+                s1 += fast_exp2(fmaf(xv[e + 1], p.scale2, neg));
+                s2 += fast_exp2(fmaf(xv[e + 2], p.scale2, neg));
+                s3 += fast_exp2(fmaf(xv[e + 3], p.scale2, neg));
               }
               sum[mb] += (s0 + s1) + (s2 + s3);
             }
           }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(TEMPTY(t));
-        }
-        // merge the two groups' partials and publish this CTA's statistics for the head
-        if (grp == 1) {
+          // merge the four column parts and publish this CTA's statistics for the head
+          if (part > 0) {
 #pragma unroll
-          for (int mb = 0; mb < 2; ++mb) merge_s[row + 128 * mb] = make_float2(mx[mb], sum[mb]);
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (grp == 0) {
-          const long long total = (long long)p.heads * p.tph;
-          const int slot = blockIdx.x - tile_owner((long long)sg.bh * p.tph, total, gridDim.x);
+            for (int mb = 0; mb < 2; ++mb) merge_s[(part - 1) * 256 + row + 128 * mb] = make_float2(mx[mb], sum[mb]);
+          }
+          asm volatile("bar.sync 1, 512;" ::: "memory");
+          if (part == 0) {
+            const long long total = (long long)p.heads * p.tph;
+            const int slot = blockIdx.x - tile_owner((long long)sg.bh * p.tph, total, gridDim.x);
 #pragma unroll
-          for (int mb = 0; mb < 2; ++mb) {
-            const int r = row + 128 * mb;
-            if (mb < p.nmblk && r < p.M) {
-              const float2 o = merge_s[r];
-              const float m = fmaxf(mx[mb], o.x);
+            for (int mb = 0; mb < 2; ++mb) {
+              const int r = row + 128 * mb;
+              if (mb < p.nmblk && r < p.M) {
+                float m = mx[mb];
+#pragma unroll
+                for (int q = 0; q < 3; ++q) m = fmaxf(m, merge_s[q * 256 + r].x);
+                float l = 0.f;
+                if (m > -INFINITY) {
+                  l = sum[mb] * fast_exp2(mx[mb] - m);
+#pragma unroll
+                  for (int q = 0; q < 3; ++q) { const float2 o = merge_s[q * 256 + r]; l += o.y * fast_exp2(o.x - m); }
+                }
+                p.stats[((size_t)sg.bh * p.slots + slot) * p.m_stride + r] = make_float2(m, l);
+              }
+            }
+          }
+          asm volatile("bar.sync 1, 512;" ::: "memory");
+        } else {
+          // ------------------------------------------------------------ sweep 2: one thread per key
+          if (sg.new_head && sid < 256) {
+            // lse2 of every window row from the partial statistics of sweep 1
+            const long long total = (long long)p.heads * p.tph;
+            const int c_lo = tile_owner((long long)sg.bh * p.tph, total, p.stats_grid);
+            const int c_hi = tile_owner((long long)(sg.bh + 1) * p.tph - 1, total, p.stats_grid);
+            float lse = INFINITY;
+            if (sid < p.M) {
+              float m = -INFINITY;
+              for (int c = 0; c <= c_hi - c_lo; ++c) m = fmaxf(m, p.stats[((size_t)sg.bh * p.slots + c) * p.m_stride + sid].x);
               float l = 0.f;
-              if (m > -INFINITY) l = sum[mb] * fast_exp2(mx[mb] - m) + o.y * fast_exp2(o.x - m);
-              p.stats[((size_t)sg.bh * p.slots + slot) * p.m_stride + r] = make_float2(m, l);
+              for (int c = 0; c <= c_hi - c_lo; ++c) {
+                const float2 st = p.stats[((size_t)sg.bh * p.slots + c) * p.m_stride + sid];
+                l += st.y * fast_exp2(st.x - m);
+              }
+              lse = m + log2f(l);
             }
+            lse_s[sid] = lse;
           }
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-      } else {
-        // ---------------------------------------------------------------- sweep 2
-        if (sg.new_head) {
-          // lse2 of every window row from the partial statistics of sweep 1
-          const long long total = (long long)p.heads * p.tph;
-          const int c_lo = tile_owner((long long)sg.bh * p.tph, total, stats_grid);
-          const int c_hi = tile_owner((long long)(sg.bh + 1) * p.tph - 1, total, stats_grid);
-          float lse = INFINITY;
-          if (sid < p.M) {
-            float m = -INFINITY;
-            for (int c = 0; c <= c_hi - c_lo; ++c) m = fmaxf(m, p.stats[((size_t)sg.bh * p.slots + c) * p.m_stride + sid].x);
-            float l = 0.f;
-            for (int c = 0; c <= c_hi - c_lo; ++c) {
-              const float2 st = p.stats[((size_t)sg.bh * p.slots + c) * p.m_stride + sid];
-              l += st.y * fast_exp2(st.x - m);
-            }
-            lse = m + log2f(l);
-          }
-          lse_s[sid] = lse;
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        for (int i = 0; i < sg.ntiles; ++i, ++tile) {
-          if ((tile & 1) != grp) continue;
-          const int t = tile & 1, nt = tile >> 1;
-          mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 107);
-          tc_fence_after();
-          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(t * stage_cols);
-          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll 1
-          for (int c = 0; c < p.nq16; c += 16) {
-            float x[16];
-            tc_ld16(taddr + c, x);
-            tc_wait_ld();
+          asm volatile("bar.sync 1, 512;" ::: "memory");
+          const int nchunk = p.nq16 >> 4;               // 16-column chunks; this warp takes part, part+4, ...
+          float* my_raw = raw_s + part * (kMaxSegTiles * kTileKeys);
+          for (int i = 0; i < sg.ntiles; ++i, ++tile) {
+            const int t = tile & 1, nt = tile >> 1;
+            mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 107);
+            tc_fence_after();
+            const uint32_t taddr = lane_addr + (uint32_t)(t * kStageCols);
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-            for (int e = 0; e < 16; e += 4) {
-              const float4 ls = *reinterpret_cast<const float4*>(&lse_s[c + e]);
-              a0 += fast_exp2(fmaf(x[e], p.scale2, -ls.x));
-              a1 += fast_exp2(fmaf(x[e + 1], p.scale2, -ls.y));
-              a2 += fast_exp2(fmaf(x[e + 2], p.scale2, -ls.z));
-              a3 += fast_exp2(fmaf(x[e + 3], p.scale2, -ls.w));
+            for (int jj = 0; jj < 2; ++jj) {                  // two 16-column chunks per round
+              const int c0 = part + 8 * jj, c1 = c0 + 4;
+              float x0[16], x1[16];
+              if (c0 < nchunk) tc_ld16(taddr + c0 * 16, x0);
+              if (c1 < nchunk) tc_ld16(taddr + c1 * 16, x1);
+              tc_wait_ld();
+              if (jj == 1 || part + 8 >= nchunk) {             // this warp's last read of the stage: release it
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(TEMPTY(t));
+              }
+              if (c0 < nchunk) {
+#pragma unroll
+                for (int e = 0; e < 16; e += 4) {
+                  const float4 ls = *reinterpret_cast<const float4*>(&lse_s[c0 * 16 + e]);
+                  a0 += fast_exp2(fmaf(x0[e], p.scale2, -ls.x));
+                  a1 += fast_exp2(fmaf(x0[e + 1], p.scale2, -ls.y));
+                  a2 += fast_exp2(fmaf(x0[e + 2], p.scale2, -ls.z));
+                  a3 += fast_exp2(fmaf(x0[e + 3], p.scale2, -ls.w));
+                }
+              }
+              if (c1 < nchunk) {
+#pragma unroll
+                for (int e = 0; e < 16; e += 4) {
+                  const float4 ls = *reinterpret_cast<const float4*>(&lse_s[c1 * 16 + e]);
+                  a0 += fast_exp2(fmaf(x1[e], p.scale2, -ls.x));
+                  a1 += fast_exp2(fmaf(x1[e + 1], p.scale2, -ls.y));
+                  a2 += fast_exp2(fmaf(x1[e + 2], p.scale2, -ls.z));
+                  a3 += fast_exp2(fmaf(x1[e + 3], p.scale2, -ls.w));
+                }
+              }
+              if (part + 8 >= nchunk) break;                   // no second round for this warp
             }
+            my_raw[i * kTileKeys + row] = (a0 + a1) + (a2 + a3);
           }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(TEMPTY(t));
-          raw_s[i * kTileKeys + row] = (a0 + a1) + (a2 + a3);
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        // Eq. 2's pooling over this segment: raw_s[x] belongs to key key0 + x
-        for (int o = sg.out0 + sid; o < sg.out1; o += kSoftmaxThreads) {
-          const int x = o - sg.key0;
-          float v = raw_s[x];
-          for (int d = 1; d <= p.half; ++d) {
-            if (o - d >= 0) v = fmaxf(v, raw_s[x - d]);
-            if (o + d < p.P) v = fmaxf(v, raw_s[x + d]);
+          asm volatile("bar.sync 1, 512;" ::: "memory");
+          // add up the four column parts in a fixed order; raw_s[x] then belongs to key key0 + x
+          for (int x = sid; x < sg.ntiles * kTileKeys; x += kSoftmaxThreads) {
+            float v = raw_s[x];
+#pragma unroll
+            for (int q = 1; q < kParts; ++q) v += raw_s[q * (kMaxSegTiles * kTileKeys) + x];
+            raw_s[x] = v;
           }
-          const size_t at = (size_t)sg.bh * p.P + o;
-          p.scores[at] = v;
-          if (p.copy_out) p.copy_out[at] = v;
+          asm volatile("bar.sync 1, 512;" ::: "memory");
+          // Eq. 2's pooling over this segment
+          for (int o = sg.out0 + sid; o < sg.out1; o += kSoftmaxThreads) {
+            const int x = o - sg.key0;
+            float v = raw_s[x];
+            for (int d = 1; d <= p.half; ++d) {
+              if (o - d >= 0) v = fmaxf(v, raw_s[x - d]);
+              if (o + d < p.P) v = fmaxf(v, raw_s[x + d]);
+            }
+            const size_t at = (size_t)sg.bh * p.P + o;
+            p.scores[at] = v;
+            if (p.copy_out) p.copy_out[at] = v;
+          }
+          asm volatile("bar.sync 1, 512;" ::: "memory");
         }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
       }
     }
   }
