@@ -120,7 +120,8 @@ int dkv_set_scores(dkv_ctx* ctx, int32_t layer, const float* scores, void* strea
  *     total order (score descending, position ascending).
  *     idx_out  : int32 [Bt, Hkv, Bl'] kept positions, ascending (optional)
  *     rank_out : int32 [Bt, Hkv, Bl'] place of each kept position in the total order, 0 = best (optional)
- *     Sets count[b][layer] = Bl'.  Needs the layer's scores (else DKV_ERR_STATE). */
+ *     Sets count[b][layer] = Bl'.  Needs the layer's scores (else DKV_ERR_STATE).  Also files the head's
+ *     scores by their leading bits for the later global top-K of dkv_rebudget. */
 int dkv_select_topk(dkv_ctx* ctx, int32_t layer, int32_t* idx_out, int32_t* rank_out, void* stream);
 
 /* (3) Eq. 4-6 / Update_Buffer_Length after `upto_layer` layers (1..L; all of them scored and selected).
@@ -133,11 +134,12 @@ int dkv_rebudget(dkv_ctx* ctx, int32_t upto_layer, int32_t* counts_out, void* st
 /* (4) Algorithm 1's buffer build and truncation for one layer.
  *     k_src, v_src != NULL : gather.  kb[b,h,0:c] = k_src[b,h,idx[0:c]], kb[b,h,c:c+ws] = k_src[b,h,P:S],
  *                            same for v; c = count[b][layer].  k_src, v_src : bf16 [Bt, Hkv, S, D].
- *     k_src == v_src == NULL : shrink kb/vb in place to the current count: rows whose rank is below
- *                            count[b][layer] stay, in position order, followed by the ws window rows.
+ *     k_src == v_src == NULL : shrink kb/vb in place to the current count: the count[b][layer] best of the
+ *                            held rows (score descending, position ascending) stay, in position order,
+ *                            followed by the ws window rows.
  *     kb, vb  : bf16 [Bt, Hkv, Bl' + ws, D] fixed stride; rows past the valid length are unspecified.
  *     len_out : int32 [Bt, Hkv] valid rows including the window (optional).
- *     The context's kept indices and ranks are compacted with the rows. */
+ *     The context's kept positions are compacted with the rows. */
 int dkv_compact(dkv_ctx* ctx, int32_t layer, const void* k_src, const void* v_src, void* kb, void* vb,
                 int32_t* len_out, void* stream);
 
@@ -161,9 +163,13 @@ int dkv_run_prefill_pass_host(dkv_ctx* ctx, const void* const* q_win, const void
 /* Copy the current counts to host int32 [Bt, L] (synchronises `stream`). */
 int dkv_get_counts(dkv_ctx* ctx, int32_t* host_counts, void* stream);
 /* Device-side views for inspection, owned by the context: the history scores of a layer
- * (fp32 [Bt,Hkv,P]) and its current kept positions / ranks (int32 [Bt,Hkv,Bl'], the first
- * held[b][layer] entries of each head valid).  Any of the out pointers may be NULL. */
-int dkv_layer_views(dkv_ctx* ctx, int32_t layer, const float** scores, const int32_t** idx, const int32_t** rank);
+ * (fp32 [Bt,Hkv,P]) and its current kept positions (int32 [Bt,Hkv,Bl'], the first held[b][layer]
+ * entries of each head valid).  Either out pointer may be NULL. */
+int dkv_layer_views(dkv_ctx* ctx, int32_t layer, const float** scores, const int32_t** idx);
+/* Rank (place in the order score descending, position ascending; 0 = best) of every position a gathered
+ * layer currently holds: rank_out int32 [Bt,Hkv,Bl'], device, first held[b][layer] entries per head
+ * written.  This is the order Algorithm 1 stores its buffers in; the buffers here are in position order. */
+int dkv_ranks(dkv_ctx* ctx, int32_t layer, int32_t* rank_out, void* stream);
 /* Device-side views of the last update's intermediate integers, int32 [Bt, L] each:
  * cnt (Eq. 4 hits per layer), Z (Eq. 5), Zp (Eq. 6), and held (rows each layer's buffers hold now). */
 int dkv_budget_views(dkv_ctx* ctx, const int32_t** cnt, const int32_t** z, const int32_t** zp, const int32_t** held);

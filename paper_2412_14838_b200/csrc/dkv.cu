@@ -26,16 +26,20 @@ struct dkv_ctx {
   // device state
   float* d_scores;      // [L][Bt][Hkv][P]  pooled scores, the history A^b
   int* d_idx;           // [L][Bt][Hkv][Blc] kept positions, ascending
-  int* d_rank;          // [L][Bt][Hkv][Blc] their ranks
   int* d_count;         // [Bt][L] budget of each layer
   int* d_held;          // [Bt][L] rows the layer's buffers hold
   int* d_dbg;           // 3 x [Bt][L] : cnt, Z, Z' of the last update
-  RbState* d_rb_state;  // [Bt]
-  unsigned int* d_rb_hist;   // [3][Bt][2048]
-  unsigned int* d_cnt_gt;    // [Bt][L]
-  unsigned int* d_cnt_eq;    // [Bt][L]
+  unsigned int* d_head_hist;  // [L][Bt][Hkv][2048] first-digit histogram of every head's scores
+  unsigned int* d_head_offs;  // [L][Bt][Hkv][2048] its ascending exclusive offsets
+  uint32_t* d_grouped;        // [L][Bt][Hkv][P] score bits grouped by first digit
+  RbState* d_rb_state;        // [Bt]
+  unsigned int* d_rb_above;   // [Bt][L]
+  unsigned int* d_rb_hist1;   // [Bt][2048]
+  unsigned int* d_rb_above2;  // [Bt][L]
+  unsigned int* d_rb_hist2;   // [Bt][L][1024]
   int* d_status;        // [8]
   int sort_n;
+  size_t shrink_smem;
   // tensor-core scoring
   int n_sms, tc_grid, tc_slots;
   float2* d_tc_stats;   // [3][Bt*Hkv][tc_slots][256]: partial softmax statistics, three layers in rotation
@@ -211,12 +215,30 @@ int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_
 }
 
 // ---- step (2): per-head top-Bl' ----------------------------------------------------------------
-int do_select(dkv_ctx* c, int layer, int* idx_out, int* rank_out, cudaStream_t st) {
+int do_ranks(dkv_ctx* c, int layer, int* rank_out, cudaStream_t st) {
   const Shape& s = c->s;
+  rank_kernel<<<s.Bt * s.Hkv, kSelThreads, (size_t)c->sort_n * 8, st>>>(
+      c->d_scores + (size_t)layer * layer_scores(s), c->d_idx + (size_t)layer * layer_idx(s), c->d_held, rank_out,
+      s.P, s.Blc, c->sort_n, s.Hkv, s.L, layer);
+  DKV_LAUNCHED(c);
+  return DKV_OK;
+}
+
+int do_select(dkv_ctx* c, int layer, int* idx_out, cudaStream_t st) {
+  const Shape& s = c->s;
+  const size_t heads = (size_t)s.Bt * s.Hkv;
   ProfScope ps(c, DKV_STEP_SELECT, 1, st);
-  select_topk_kernel<<<s.Bt * s.Hkv, kSelThreads, (size_t)c->sort_n * 8, st>>>(
-      c->d_scores + (size_t)layer * layer_scores(s), c->d_idx + (size_t)layer * layer_idx(s),
-      c->d_rank + (size_t)layer * layer_idx(s), idx_out, rank_out, s.P, s.Blc, c->sort_n, c->d_count, s.Hkv, s.L, layer);
+  const float* sc = c->d_scores + (size_t)layer * layer_scores(s);
+  int* idx = c->d_idx + (size_t)layer * layer_idx(s);
+  unsigned int* hh = c->d_head_hist + (size_t)layer * heads * kBins;
+  unsigned int* ho = c->d_head_offs + (size_t)layer * heads * kBins;
+  uint32_t* gr = c->d_grouped + (size_t)layer * layer_scores(s);
+  if ((s.P + kSelThreads - 1) / kSelThreads <= kRegChunk)
+    select_topk_kernel<true><<<(unsigned)heads, kSelThreads, 0, st>>>(sc, idx, idx_out, hh, ho, gr, s.P, s.Blc, c->d_count,
+                                                                     s.Hkv, s.L, layer);
+  else
+    select_topk_kernel<false><<<(unsigned)heads, kSelThreads, 0, st>>>(sc, idx, idx_out, hh, ho, gr, s.P, s.Blc, c->d_count,
+                                                                      s.Hkv, s.L, layer);
   DKV_LAUNCHED(c);
   c->selected[layer] = 1;
   c->gathered[layer] = c->stale[layer] = 0;
@@ -226,30 +248,24 @@ int do_select(dkv_ctx* c, int layer, int* idx_out, int* rank_out, cudaStream_t s
 // ---- step (3): Update_Buffer_Length ------------------------------------------------------------
 int do_rebudget(dkv_ctx* c, int l, int* counts_out, cudaStream_t st) {
   const Shape& s = c->s;
-  const size_t per_layer = (size_t)s.Hkv * s.P;
   long long k = (long long)s.N * s.Hkv * l;
-  const long long pop = (long long)l * (long long)per_layer;
+  const long long pop = (long long)l * s.Hkv * s.P;
   if (k > pop) k = pop;
-  ProfScope ps(c, DKV_STEP_REBUDGET, 9, st);
-  const int init_n = 3 * s.Bt * kRbBins > s.Bt * s.L ? 3 * s.Bt * kRbBins : s.Bt * s.L;
-  rb_init_kernel<<<(init_n + 255) / 256, 256, 0, st>>>(c->d_rb_state, c->d_rb_hist, c->d_cnt_gt, c->d_cnt_eq, s.Bt, s.L,
-                                                      (unsigned int)k);
+  ProfScope ps(c, DKV_STEP_REBUDGET, 4, st);
+  rb_locate_kernel<<<s.Bt, 1024, 0, st>>>(c->d_head_hist, c->d_head_offs, c->d_rb_state, c->d_rb_above, c->d_rb_hist1,
+                                         c->d_rb_above2, c->d_rb_hist2, s.Bt, s.Hkv, s.L, l, s.P, k);
   DKV_LAUNCHED(c);
-  int bpl = (int)((per_layer + (size_t)kRbThreads * 8 - 1) / ((size_t)kRbThreads * 8));
-  if (bpl > 64) bpl = 64;
-  if (bpl < 1) bpl = 1;
-  const dim3 grid(bpl, l, s.Bt);
-  for (int pass = 0; pass < 3; ++pass) {
-    rb_hist_kernel<<<grid, kRbThreads, 0, st>>>(c->d_scores, c->d_rb_state, c->d_rb_hist, pass, s.Bt, per_layer);
-    DKV_LAUNCHED(c);
-    rb_scan_kernel<<<s.Bt, 1024, 0, st>>>(c->d_rb_state, c->d_rb_hist, pass, s.Bt);
-    DKV_LAUNCHED(c);
-  }
-  rb_count_kernel<<<grid, kRbThreads, 0, st>>>(c->d_scores, c->d_rb_state, c->d_cnt_gt, c->d_cnt_eq, s.Bt, s.L, per_layer);
+  const dim3 grid(4, l * s.Hkv, s.Bt);
+  rb_refine1_kernel<<<grid, kRbThreads, 0, st>>>(c->d_grouped, c->d_head_hist, c->d_head_offs, c->d_rb_state,
+                                                c->d_rb_hist1, s.Bt, s.Hkv, s.P);
+  DKV_LAUNCHED(c);
+  rb_refine2_kernel<<<grid, kRbThreads, 0, st>>>(c->d_grouped, c->d_head_hist, c->d_head_offs, c->d_rb_state,
+                                                c->d_rb_hist1, c->d_rb_above2, c->d_rb_hist2, s.Bt, s.Hkv, s.L, s.P);
   DKV_LAUNCHED(c);
   const size_t bl = (size_t)s.Bt * s.L;
-  rb_budget_kernel<<<(s.Bt + 31) / 32, 32, 0, st>>>(c->d_cnt_gt, c->d_cnt_eq, c->d_count, c->d_dbg, c->d_dbg + bl,
-                                                   c->d_dbg + 2 * bl, counts_out, s.Bt, s.L, l, k, s.Bl, s.N);
+  rb_budget_kernel<<<s.Bt, 1024, 0, st>>>(c->d_rb_state, c->d_rb_hist1, c->d_rb_above, c->d_rb_above2, c->d_rb_hist2,
+                                         c->d_count, c->d_dbg, c->d_dbg + bl, c->d_dbg + 2 * bl, counts_out, s.Bt, s.L, l,
+                                         s.Bl, s.N);
   DKV_LAUNCHED(c);
   for (int i = 0; i < l; ++i) if (!c->gathered[i]) c->stale[i] = 1;
   return DKV_OK;
@@ -261,9 +277,9 @@ int do_shrink(dkv_ctx* c, int layer0, int n, void* const* kb, void* const* vb, c
   LayerPtrs ptrs;
   for (int i = 0; i < n; ++i) { ptrs.kb[layer0 + i] = kb[i]; ptrs.vb[layer0 + i] = vb[i]; }
   ProfScope ps(c, DKV_STEP_SHRINK, 2, st);
-  shrink_kernel<<<dim3(s.Bt * s.Hkv, n), kShrinkThreads, (size_t)s.Blc * 4, st>>>(
-      ptrs, layer0, c->d_idx, c->d_rank, c->d_count, c->d_held, s.Bt, s.Hkv, s.L, s.ws, s.Blc, s.rows, s.D * 2 / 16,
-      layer_idx(s));
+  shrink_kernel<<<dim3(s.Bt * s.Hkv, n), kShrinkThreads, c->shrink_smem, st>>>(
+      ptrs, layer0, c->d_scores, c->d_idx, c->d_count, c->d_held, s.Bt, s.Hkv, s.L, s.P, s.ws, s.Blc, s.rows,
+      s.D * 2 / 16, layer_idx(s), layer_scores(s));
   DKV_LAUNCHED(c);
   commit_held_kernel<<<(s.Bt * n + 127) / 128, 128, 0, st>>>(c->d_held, c->d_count, s.Bt, s.L, layer0, n);
   DKV_LAUNCHED(c);
@@ -272,7 +288,7 @@ int do_shrink(dkv_ctx* c, int layer0, int n, void* const* kb, void* const* vb, c
 
 int do_gather(dkv_ctx* c, int layer, const void* k_src, const void* v_src, void* kb, void* vb, cudaStream_t st) {
   const Shape& s = c->s;
-  const int vec = s.D * 2 / 16, rpb = 256 / vec;
+  const int vec = s.D * 2 / 16, rpb = 256 / vec * kGatherRows;
   const dim3 grid((s.rows + rpb - 1) / rpb, s.Bt * s.Hkv, 2);
   {
   ProfScope ps(c, DKV_STEP_GATHER, 1, st);
@@ -323,7 +339,7 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
     c->scored[el] = 1;
     DKV_CUDA(c, cudaEventRecord(c->ev_scored[el], st));
     DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_scored[el], 0));
-    if ((rc = do_select(c, el, nullptr, nullptr, sd))) return rc;
+    if ((rc = do_select(c, el, nullptr, sd))) return rc;
     if ((rc = do_gather(c, el, k[el], v[el], kb[el], vb[el], sd))) return rc;
     const bool update = ((el + 1) % s.m == 0) || (el + 1 == s.L && s.L % s.m != 0);
     if (update) {
@@ -337,9 +353,10 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
 }
 
 void free_all(dkv_ctx* c) {
-  cudaFree(c->d_scores); cudaFree(c->d_idx); cudaFree(c->d_rank); cudaFree(c->d_count);
-  cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_rb_state); cudaFree(c->d_rb_hist);
-  cudaFree(c->d_cnt_gt); cudaFree(c->d_cnt_eq); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
+  cudaFree(c->d_scores); cudaFree(c->d_idx); cudaFree(c->d_count);
+  cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_rb_state); cudaFree(c->d_rb_above); cudaFree(c->d_rb_hist1);
+  cudaFree(c->d_rb_above2); cudaFree(c->d_rb_hist2); cudaFree(c->d_head_hist); cudaFree(c->d_head_offs);
+  cudaFree(c->d_grouped); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
   if (c->side) cudaStreamDestroy(c->side);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
@@ -425,7 +442,12 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
     c->n_sms = sms > 0 ? sms : 1;
     const int tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
     const long long total_tiles = (long long)heads * tph;
-    c->tc_grid = (int)(total_tiles < c->n_sms ? total_tiles : c->n_sms);
+    // leave a few SMs to the per-head select CTAs that dkv_run_prefill_pass runs beside the scoring
+    int side = heads < c->n_sms / 8 ? heads : c->n_sms / 8;
+    if (const char* e = getenv("DKV_SIDE_SMS")) side = atoi(e);
+    int score_sms = c->n_sms - side;
+    if (score_sms < 1) score_sms = 1;
+    c->tc_grid = (int)(total_tiles < score_sms ? total_tiles : score_sms);
     int slots = 1;
     for (int bh = 0; bh < heads; ++bh) {
       const int lo = tc::tile_owner((long long)bh * tph, total_tiles, c->tc_grid);
@@ -438,14 +460,17 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
 #define TRY(call) if (e == cudaSuccess) e = (call)
   TRY(cudaMalloc(&c->d_scores, sizeof(float) * s.L * layer_scores(s)));
   TRY(cudaMalloc(&c->d_idx, sizeof(int) * s.L * layer_idx(s)));
-  TRY(cudaMalloc(&c->d_rank, sizeof(int) * s.L * layer_idx(s)));
   TRY(cudaMalloc(&c->d_count, sizeof(int) * bl));
   TRY(cudaMalloc(&c->d_held, sizeof(int) * bl));
   TRY(cudaMalloc(&c->d_dbg, sizeof(int) * 3 * bl));
   TRY(cudaMalloc(&c->d_rb_state, sizeof(RbState) * s.Bt));
-  TRY(cudaMalloc(&c->d_rb_hist, sizeof(unsigned int) * 3 * s.Bt * kRbBins));
-  TRY(cudaMalloc(&c->d_cnt_gt, sizeof(unsigned int) * bl));
-  TRY(cudaMalloc(&c->d_cnt_eq, sizeof(unsigned int) * bl));
+  TRY(cudaMalloc(&c->d_rb_above, sizeof(unsigned int) * bl));
+  TRY(cudaMalloc(&c->d_rb_above2, sizeof(unsigned int) * bl));
+  TRY(cudaMalloc(&c->d_rb_hist1, sizeof(unsigned int) * s.Bt * kBins));
+  TRY(cudaMalloc(&c->d_rb_hist2, sizeof(unsigned int) * bl * 1024));
+  TRY(cudaMalloc(&c->d_head_hist, sizeof(unsigned int) * s.L * heads * kBins));
+  TRY(cudaMalloc(&c->d_head_offs, sizeof(unsigned int) * s.L * heads * kBins));
+  TRY(cudaMalloc(&c->d_grouped, sizeof(uint32_t) * s.L * layer_scores(s)));
   TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * 3 * heads * c->tc_slots * 256));
   TRY(cudaFuncSetAttribute(tc::score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   TRY(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
@@ -457,8 +482,9 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMemset(c->d_count, 0, sizeof(int) * bl));
   TRY(cudaMemset(c->d_held, 0, sizeof(int) * bl));
   TRY(cudaMemset(c->d_dbg, 0, sizeof(int) * 3 * bl));
-  TRY(cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, c->sort_n * 8));
-  TRY(cudaFuncSetAttribute(shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, s.Blc * 4));
+  c->shrink_smem = sizeof(int) * (size_t)(s.Blc > kBins ? s.Blc : kBins);
+  TRY(cudaFuncSetAttribute(rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, c->sort_n * 8));
+  TRY(cudaFuncSetAttribute(shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->shrink_smem));
 #undef TRY
   if (e != cudaSuccess) {
     rc = e == cudaErrorMemoryAllocation ? DKV_ERR_NOMEM : DKV_ERR_CUDA;
@@ -507,7 +533,15 @@ int dkv_select_topk(dkv_ctx* c, int32_t layer, int32_t* idx_out, int32_t* rank_o
   int rc = check_layer(c, layer);
   if (rc) return rc;
   if (!c->scored[layer]) return DKV_ERR_STATE;
-  return do_select(c, layer, idx_out, rank_out, as_stream(stream));
+  rc = do_select(c, layer, idx_out, as_stream(stream));
+  if (rc || !rank_out) return rc;
+  // ranks of a fresh selection: every head holds Bl' positions
+  const Shape& s = c->s;
+  rank_kernel<<<s.Bt * s.Hkv, kSelThreads, (size_t)c->sort_n * 8, as_stream(stream)>>>(
+      c->d_scores + (size_t)layer * layer_scores(s), c->d_idx + (size_t)layer * layer_idx(s), c->d_count, rank_out,
+      s.P, s.Blc, c->sort_n, s.Hkv, s.L, layer);
+  DKV_LAUNCHED(c);
+  return DKV_OK;
 }
 
 int dkv_rebudget(dkv_ctx* c, int32_t upto_layer, int32_t* counts_out, void* stream) {
@@ -579,7 +613,7 @@ int dkv_run_prefill_pass_host(dkv_ctx* c, const void* const* q_win, const void* 
     DKV_CUDA(c, cudaEventRecord(c->ev_copied[slot], cp));
     DKV_CUDA(c, cudaStreamWaitEvent(st, c->ev_copied[slot], 0));
     if ((rc = do_score(c, l, c->st_q[slot], c->st_k[slot], nullptr, st))) return rc;
-    if ((rc = do_select(c, l, nullptr, nullptr, st))) return rc;
+    if ((rc = do_select(c, l, nullptr, st))) return rc;
     if ((rc = do_gather(c, l, c->st_k[slot], c->st_v[slot], c->st_kb[l], c->st_vb[l], st))) return rc;
     DKV_CUDA(c, cudaEventRecord(c->ev_consumed[slot], st));
     const bool update = ((l + 1) % s.m == 0) || (l + 1 == s.L && s.L % s.m != 0);
@@ -607,13 +641,20 @@ int dkv_get_counts(dkv_ctx* c, int32_t* host_counts, void* stream) {
   return DKV_OK;
 }
 
-int dkv_layer_views(dkv_ctx* c, int32_t layer, const float** scores, const int32_t** idx, const int32_t** rank) {
+int dkv_layer_views(dkv_ctx* c, int32_t layer, const float** scores, const int32_t** idx) {
   int rc = check_layer(c, layer);
   if (rc) return rc;
   if (scores) *scores = c->d_scores + (size_t)layer * layer_scores(c->s);
   if (idx) *idx = c->d_idx + (size_t)layer * layer_idx(c->s);
-  if (rank) *rank = c->d_rank + (size_t)layer * layer_idx(c->s);
   return DKV_OK;
+}
+
+int dkv_ranks(dkv_ctx* c, int32_t layer, int32_t* rank_out, void* stream) {
+  int rc = check_layer(c, layer);
+  if (rc) return rc;
+  if (!rank_out) return DKV_ERR_INVALID_ARG;
+  if (!c->gathered[layer]) return DKV_ERR_STATE;
+  return do_ranks(c, layer, rank_out, as_stream(stream));
 }
 
 int dkv_budget_views(dkv_ctx* c, const int32_t** cnt, const int32_t** z, const int32_t** zp, const int32_t** held) {

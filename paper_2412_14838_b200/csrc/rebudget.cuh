@@ -1,151 +1,191 @@
-// Update_Buffer_Length (Eq. 4-6) on the device: a global top-K over the score history of the
-// layers processed so far, counted per layer, then the integer budget arithmetic.
-// Only per-layer counts leave the selection, so the K-th largest value T is found by a 3-pass
-// radix select on the scores' bit patterns (non-negative floats order like unsigned ints), and
-// the entries equal to T are handed out in flat-index order, i.e. to the lowest layers first.
+// Update_Buffer_Length (Eq. 4-6) on the device: the K-th largest of all scores of the layers processed
+// so far, the number of top-K hits per layer, then the integer budget arithmetic.
+//
+// Only per-layer counts leave the selection.  Every head's scores were histogrammed by their first
+// 11-bit digit and stored grouped by that digit when the layer was selected (select.cuh), so:
+//   rb_locate   adds up the per-head histograms of layers [0, l), finds the digit b* that holds the K-th
+//               largest score, and reads each layer's count of scores above b* off the offsets;
+//   rb_refine1  histograms the next 11 bits of the scores inside bucket b* (the only scores read);
+//   rb_refine2  counts, per layer, the bucket's scores above the second digit and histograms the last
+//               10 bits of those that match it;
+//   rb_budget   fixes the exact threshold T, gives the entries equal to T to the lowest layers first
+//               (flat-index tie rule), and evaluates Eq. 5-6 in exact integers.
 #pragma once
 #include "common.cuh"
+#include "select.cuh"
 
 namespace dkv {
 
-constexpr int kRbBins = 2048;
-constexpr int kRbThreads = 512;
+constexpr int kRbThreads = 256;
 
 struct RbState {          // per sample
-  uint32_t prefix, mask;
-  uint32_t remaining;     // how many of the entries matching `prefix` are still to be taken
-  uint32_t pad;
+  int bstar;              // first digit of T
+  int need1;              // entries still to take inside bucket b*
+  int cand;               // entries in bucket b* over all layers and heads
+  int pad;
 };
 
-__device__ __forceinline__ int rb_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
-__device__ __forceinline__ uint32_t rb_bins(int pass) { return pass == 2 ? 1024u : 2048u; }
-
-// Start of an update: clear histograms and per-layer counters, state = (no prefix, k to take).
-__global__ void rb_init_kernel(RbState* __restrict__ state, unsigned int* __restrict__ hist, unsigned int* __restrict__ cnt_gt,
-                               unsigned int* __restrict__ cnt_eq, int Bt, int L, unsigned int k) {
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e < 3 * Bt * kRbBins) hist[e] = 0;
-  if (e < Bt * L) { cnt_gt[e] = 0; cnt_eq[e] = 0; }
-  if (e < Bt) { RbState st; st.prefix = 0; st.mask = 0; st.remaining = k; st.pad = 0; state[e] = st; }
-}
-
-// History layout: scores[layer][b][h][p].  grid (blocks per layer, l, Bt).
-__global__ void __launch_bounds__(kRbThreads)
-rb_hist_kernel(const float* __restrict__ scores, const RbState* __restrict__ state, unsigned int* __restrict__ hist,
-               int pass, int Bt, size_t per_layer /* Hkv*P */) {
-  __shared__ unsigned int sh[kRbBins];
-  const int b = blockIdx.z, layer = blockIdx.y;
-  for (int i = threadIdx.x; i < kRbBins; i += kRbThreads) sh[i] = 0;
-  __syncthreads();
-  const RbState st = state[b];
-  const int shift = rb_shift(pass);
-  const uint32_t bmask = rb_bins(pass) - 1u;
-  const uint32_t* v = reinterpret_cast<const uint32_t*>(scores) + ((size_t)layer * Bt + b) * per_layer;
-  for (size_t i = (size_t)blockIdx.x * kRbThreads + threadIdx.x; i < per_layer; i += (size_t)gridDim.x * kRbThreads) {
-    const uint32_t u = v[i];
-    if ((u & st.mask) == st.prefix) atomicAdd(&sh[(u >> shift) & bmask], 1u);
-  }
-  __syncthreads();
-  unsigned int* gh = hist + ((size_t)pass * Bt + b) * kRbBins;
-  for (int i = threadIdx.x; i < kRbBins; i += kRbThreads) {
-    const unsigned int c = sh[i];
-    if (c) atomicAdd(&gh[i], c);
-  }
-}
-
-// One block per sample: locate the bin holding the `remaining`-th largest entry and narrow the prefix.
+// One CTA of 1024 threads per sample.
+// head_hist/head_offs: [L][Bt][Hkv][2048].  above: [Bt][L] scores above bucket b* per layer.
+// hist1: [Bt][2048], above2: [Bt][L], hist2: [Bt][L][1024] are cleared here for the refine kernels.
 __global__ void __launch_bounds__(1024)
-rb_scan_kernel(RbState* __restrict__ state, const unsigned int* __restrict__ hist, int pass, int Bt) {
-  __shared__ unsigned int cum[kRbBins];
-  const int b = blockIdx.x;
-  const unsigned int* gh = hist + ((size_t)pass * Bt + b) * kRbBins;
-  for (int i = threadIdx.x; i < kRbBins; i += blockDim.x) cum[i] = gh[i];
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    RbState st = state[b];
-    unsigned int above = 0;
-    int bin = (int)rb_bins(pass) - 1;
-    for (; bin > 0; --bin) {
-      const unsigned int c = cum[bin];
-      if (above + c >= st.remaining) break;
-      above += c;
+rb_locate_kernel(const unsigned int* __restrict__ head_hist, const unsigned int* __restrict__ head_offs,
+                 RbState* __restrict__ state, unsigned int* __restrict__ above, unsigned int* __restrict__ hist1,
+                 unsigned int* __restrict__ above2, unsigned int* __restrict__ hist2,
+                 int Bt, int Hkv, int L, int l, int P, long long k) {
+  __shared__ unsigned int hist[kBins];
+  __shared__ int sm_scan[33];
+  __shared__ int found[2];
+  const int b = blockIdx.x, tid = threadIdx.x;
+  for (int bin = tid; bin < kBins; bin += 1024) {
+    unsigned int s = 0;
+    for (int ih = 0; ih < l * Hkv; ++ih) {
+      const int i = ih / Hkv, h = ih % Hkv;
+      s += head_hist[(((size_t)i * Bt + b) * Hkv + h) * kBins + bin];
     }
-    const int shift = rb_shift(pass);
-    st.prefix |= ((uint32_t)bin) << shift;
-    st.mask |= (rb_bins(pass) - 1u) << shift;
-    st.remaining -= above;
-    state[b] = st;
+    hist[bin] = s;
+    hist1[(size_t)b * kBins + bin] = 0;
+  }
+  for (int e = tid; e < L; e += 1024) above2[b * L + e] = 0;
+  for (int e = tid; e < l * 1024; e += 1024) hist2[(size_t)b * L * 1024 + e] = 0;
+  __syncthreads();
+  const long long total = (long long)l * Hkv * P;
+  find_digit(hist, kBins, (int)total, (int)k, sm_scan, found, nullptr);
+  const int d = found[0];
+  if (tid == 0) { RbState st; st.bstar = d; st.need1 = found[1]; st.cand = (int)hist[d]; st.pad = 0; state[b] = st; }
+  for (int i = tid; i < l; i += 1024) {
+    unsigned int a = 0;
+    for (int h = 0; h < Hkv; ++h) {
+      const size_t at = (((size_t)i * Bt + b) * Hkv + h) * kBins + d;
+      a += (unsigned int)P - head_offs[at] - head_hist[at];
+    }
+    above[b * L + i] = a;
   }
 }
 
-// Per (layer, sample): entries above T and entries equal to T.  grid (blocks per layer, l, Bt).
+// grid (slices, l * Hkv, Bt): second-digit histogram of the scores in bucket b*.
 __global__ void __launch_bounds__(kRbThreads)
-rb_count_kernel(const float* __restrict__ scores, const RbState* __restrict__ state, unsigned int* __restrict__ cnt_gt,
-                unsigned int* __restrict__ cnt_eq, int Bt, int L, size_t per_layer) {
-  __shared__ unsigned int s_gt[kRbThreads / 32], s_eq[kRbThreads / 32];
-  const int b = blockIdx.z, layer = blockIdx.y;
-  const uint32_t T = state[b].prefix;
-  const uint32_t* v = reinterpret_cast<const uint32_t*>(scores) + ((size_t)layer * Bt + b) * per_layer;
-  unsigned int gt = 0, eq = 0;
-  for (size_t i = (size_t)blockIdx.x * kRbThreads + threadIdx.x; i < per_layer; i += (size_t)gridDim.x * kRbThreads) {
-    const uint32_t u = v[i];
-    gt += (u > T); eq += (u == T);
+rb_refine1_kernel(const uint32_t* __restrict__ grouped, const unsigned int* __restrict__ head_hist,
+                  const unsigned int* __restrict__ head_offs, const RbState* __restrict__ state,
+                  unsigned int* __restrict__ hist1, int Bt, int Hkv, int P) {
+  __shared__ unsigned int sh[kBins];
+  const int b = blockIdx.z, i = blockIdx.y / Hkv, h = blockIdx.y % Hkv;
+  const int d = state[b].bstar;
+  const size_t head = ((size_t)i * Bt + b) * Hkv + h;
+  const int n = (int)head_hist[head * kBins + d];
+  if ((int)(blockIdx.x * kRbThreads) >= n) return;
+  const uint32_t* src = grouped + head * P + head_offs[head * kBins + d];
+  for (int j = threadIdx.x; j < kBins; j += kRbThreads) sh[j] = 0;
+  __syncthreads();
+  for (int e = blockIdx.x * kRbThreads + threadIdx.x; e < n; e += gridDim.x * kRbThreads)
+    atomicAdd(&sh[(src[e] >> 10) & 2047u], 1u);
+  __syncthreads();
+  for (int j = threadIdx.x; j < kBins; j += kRbThreads) { const unsigned int c = sh[j]; if (c) atomicAdd(&hist1[(size_t)b * kBins + j], c); }
+}
+
+// Same grid.  Every block re-derives the second digit s* from hist1; then per layer: bucket scores with a
+// larger second digit (above2) and the last-10-bit histogram of those with second digit s* (hist2).
+__global__ void __launch_bounds__(kRbThreads)
+rb_refine2_kernel(const uint32_t* __restrict__ grouped, const unsigned int* __restrict__ head_hist,
+                  const unsigned int* __restrict__ head_offs, const RbState* __restrict__ state,
+                  const unsigned int* __restrict__ hist1, unsigned int* __restrict__ above2,
+                  unsigned int* __restrict__ hist2, int Bt, int Hkv, int L, int P) {
+  __shared__ unsigned int sh[kBins];
+  __shared__ int sm_scan[33];
+  __shared__ int found[2];
+  __shared__ unsigned int s_above;
+  const int b = blockIdx.z, i = blockIdx.y / Hkv, h = blockIdx.y % Hkv;
+  const RbState st = state[b];
+  const size_t head = ((size_t)i * Bt + b) * Hkv + h;
+  const int n = (int)head_hist[head * kBins + st.bstar];
+  if ((int)(blockIdx.x * kRbThreads) >= n) return;
+  for (int j = threadIdx.x; j < kBins; j += kRbThreads) sh[j] = hist1[(size_t)b * kBins + j];
+  if (threadIdx.x == 0) s_above = 0;
+  __syncthreads();
+  find_digit(sh, kBins, st.cand, st.need1, sm_scan, found, nullptr);
+  const uint32_t s2 = (uint32_t)found[0];
+  const uint32_t* src = grouped + head * P + head_offs[head * kBins + st.bstar];
+  unsigned int mine = 0;
+  for (int e = blockIdx.x * kRbThreads + threadIdx.x; e < n; e += gridDim.x * kRbThreads) {
+    const uint32_t u = src[e], dd = (u >> 10) & 2047u;
+    if (dd > s2) ++mine;
+    else if (dd == s2) atomicAdd(&hist2[((size_t)b * L + i) * 1024 + (u & 1023u)], 1u);
   }
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    gt += __shfl_xor_sync(0xFFFFFFFFu, gt, o);
-    eq += __shfl_xor_sync(0xFFFFFFFFu, eq, o);
-  }
-  if ((threadIdx.x & 31) == 0) { s_gt[threadIdx.x >> 5] = gt; s_eq[threadIdx.x >> 5] = eq; }
+  for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
+  if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&s_above, mine);
   __syncthreads();
-  if (threadIdx.x == 0) {
-    unsigned int g = 0, e = 0;
-    for (int w = 0; w < kRbThreads / 32; ++w) { g += s_gt[w]; e += s_eq[w]; }
-    if (g) atomicAdd(&cnt_gt[b * L + layer], g);
-    if (e) atomicAdd(&cnt_eq[b * L + layer], e);
-  }
+  if (threadIdx.x == 0 && s_above) atomicAdd(&above2[b * L + i], s_above);
 }
 
-// Eq. 5-6 in exact integers, one thread per sample (at most 128 layers).
-// cnt_i = gt_i + share of the ties; Z_i = floor(Bl*cnt_i/max cnt); Z'_i = floor(Z_i*N*L/sum Z);
-// count_i = min(count_i, Z'_i).
-__global__ void rb_budget_kernel(const unsigned int* __restrict__ cnt_gt, const unsigned int* __restrict__ cnt_eq,
-                                 int* __restrict__ count, int* __restrict__ dbg_cnt, int* __restrict__ dbg_z,
-                                 int* __restrict__ dbg_zp, int* __restrict__ counts_out,
-                                 int Bt, int L, int l, long long k, int Bl, int N) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= Bt) return;
-  long long above = 0;
-  for (int i = 0; i < l; ++i) above += cnt_gt[b * L + i];
-  long long need = k - above;             // ties still to hand out, lowest layers first
-  long long cmax = 0;
-  for (int i = 0; i < l; ++i) {
-    const long long e = cnt_eq[b * L + i];
-    long long take = need < e ? need : e;
-    if (take < 0) take = 0;
-    need -= take;
-    const long long c = (long long)cnt_gt[b * L + i] + take;
-    dbg_cnt[b * L + i] = (int)c;
-    cmax = c > cmax ? c : cmax;
+// One CTA of 1024 threads per sample: exact T, per-layer hits, Eq. 5-6.
+// cnt_i = hits of layer i among the K largest (ties at T to the lowest layers first);
+// Z_i = floor(Bl*cnt_i/max cnt); Z'_i = floor(Z_i*N*L/sum Z); count_i = min(count_i, Z'_i).
+__global__ void __launch_bounds__(1024)
+rb_budget_kernel(const RbState* __restrict__ state, const unsigned int* __restrict__ hist1,
+                 const unsigned int* __restrict__ above, const unsigned int* __restrict__ above2,
+                 const unsigned int* __restrict__ hist2, int* __restrict__ count, int* __restrict__ dbg_cnt,
+                 int* __restrict__ dbg_z, int* __restrict__ dbg_zp, int* __restrict__ counts_out,
+                 int Bt, int L, int l, int Bl, int N) {
+  __shared__ unsigned int sh[kBins];
+  __shared__ int sm_scan[33];
+  __shared__ int found[2];
+  __shared__ long long s_gt[128], s_eq[128];
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const RbState st = state[b];
+  for (int j = tid; j < kBins; j += 1024) sh[j] = hist1[(size_t)b * kBins + j];
+  __syncthreads();
+  find_digit(sh, kBins, st.cand, st.need1, sm_scan, found, nullptr);
+  const int need2 = found[1];
+  const int cand2 = (int)sh[found[0]];
+  __syncthreads();
+  // last digit: total histogram over layers
+  for (int j = tid; j < kBins; j += 1024) {
+    unsigned int s = 0;
+    if (j < 1024) for (int i = 0; i < l; ++i) s += hist2[((size_t)b * L + i) * 1024 + j];
+    sh[j] = s;
   }
-  if (cmax <= 0) cmax = 1;
-  long long sumz = 0;
-  for (int i = 0; i < l; ++i) {
-    const long long z = ((long long)Bl * dbg_cnt[b * L + i]) / cmax;
-    dbg_z[b * L + i] = (int)z;
-    sumz += z;
+  __syncthreads();
+  find_digit(sh, kBins, cand2, need2, sm_scan, found, nullptr);
+  const int t_low = found[0];
+  long long ties = found[1];                  // entries equal to T that are taken, lowest layers first
+  // per layer: entries above T and equal to T (one warp per layer)
+  for (int i = warp; i < l; i += 32) {
+    unsigned int g = 0;
+    for (int j = t_low + 1 + lane; j < 1024; j += 32) g += hist2[((size_t)b * L + i) * 1024 + j];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) g += __shfl_xor_sync(0xFFFFFFFFu, g, o);
+    if (lane == 0) {
+      s_gt[i] = (long long)above[b * L + i] + above2[b * L + i] + g;
+      s_eq[i] = hist2[((size_t)b * L + i) * 1024 + t_low];
+    }
   }
-  if (sumz <= 0) sumz = 1;
-  const long long B = (long long)N * L;
-  for (int i = 0; i < l; ++i) {
-    const long long zp = ((long long)dbg_z[b * L + i] * B) / sumz;
-    const int zpi = zp > 0x7FFFFFFF ? 0x7FFFFFFF : (int)zp;
-    dbg_zp[b * L + i] = zpi;
-    const int c = count[b * L + i];
-    count[b * L + i] = c < zpi ? c : zpi;
+  __syncthreads();
+  if (tid == 0) {
+    long long cmax = 0;
+    for (int i = 0; i < l; ++i) {
+      const long long take = ties < s_eq[i] ? ties : s_eq[i];
+      ties -= take;
+      s_gt[i] += take;                        // = cnt_i
+      dbg_cnt[b * L + i] = (int)s_gt[i];
+      cmax = s_gt[i] > cmax ? s_gt[i] : cmax;
+    }
+    if (cmax <= 0) cmax = 1;
+    long long sumz = 0;
+    for (int i = 0; i < l; ++i) { s_eq[i] = ((long long)Bl * s_gt[i]) / cmax; dbg_z[b * L + i] = (int)s_eq[i]; sumz += s_eq[i]; }
+    if (sumz <= 0) sumz = 1;
+    const long long B = (long long)N * L;
+    for (int i = 0; i < l; ++i) {
+      const long long zp = (s_eq[i] * B) / sumz;
+      const int zpi = zp > 0x7FFFFFFF ? 0x7FFFFFFF : (int)zp;
+      dbg_zp[b * L + i] = zpi;
+      const int c = count[b * L + i];
+      count[b * L + i] = c < zpi ? c : zpi;
+    }
+    for (int i = l; i < L; ++i) { dbg_cnt[b * L + i] = 0; dbg_z[b * L + i] = 0; dbg_zp[b * L + i] = 0; }
   }
-  for (int i = l; i < L; ++i) { dbg_cnt[b * L + i] = 0; dbg_z[b * L + i] = 0; dbg_zp[b * L + i] = 0; }
-  if (counts_out) for (int i = 0; i < L; ++i) counts_out[b * L + i] = count[b * L + i];
+  __syncthreads();
+  if (counts_out) for (int i = tid; i < L; i += 1024) counts_out[b * L + i] = count[b * L + i];
 }
 
 }  // namespace dkv

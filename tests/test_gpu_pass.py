@@ -65,8 +65,11 @@ class GpuPass:
 
     def idx_rank(self, layer):
         w = self.w
-        _, ia, ra = B.dkv_layer_views(self.h, layer)
-        return (B.read_device_i32(self.h, ia, (w.Bt, w.Hkv, w.Blc)), B.read_device_i32(self.h, ra, (w.Bt, w.Hkv, w.Blc)))
+        _, ia = B.dkv_layer_views(self.h, layer)
+        rank = torch.zeros((w.Bt, w.Hkv, w.Blc), dtype=torch.int32, device="cuda")
+        B.dkv_ranks(self.h, layer, rank)
+        torch.cuda.synchronize()
+        return B.read_device_i32(self.h, ia, (w.Bt, w.Hkv, w.Blc)), rank.cpu().numpy()
 
     def close(self):
         B.dkv_destroy(self.h)

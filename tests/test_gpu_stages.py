@@ -69,7 +69,7 @@ def test_score_matches_oracle(w):
             ref = O.window_scores(synth.bf16_bits_to_f64(t["q"]), synth.bf16_bits_to_f64(t["k"]), w.ws, w.pool)["score"]
             U.assert_scores_close(got, ref, f"{w.name} layer {layer}")
             # the history slot holds the same values as the copy-out
-            addr, _, _ = B.dkv_layer_views(c.h, layer)
+            addr, _ = B.dkv_layer_views(c.h, layer)
             hist = np.empty_like(got)
             B.dkv_memcpy_to_host(c.h, hist, addr, hist.nbytes)
             assert (hist == got).all()
@@ -245,9 +245,12 @@ def test_gather_and_shrink_bytes(D):
         for l in range(w.L):
             got_k = kb[l].cpu().numpy().view(np.uint16)
             got_v = vb[l].cpu().numpy().view(np.uint16)
-            _, idx_a, rank_a = B.dkv_layer_views(c.h, l)
+            _, idx_a = B.dkv_layer_views(c.h, l)
             idx_now = B.read_device_i32(c.h, idx_a, (w.Bt, w.Hkv, w.Blc))
-            rank_now = B.read_device_i32(c.h, rank_a, (w.Bt, w.Hkv, w.Blc))
+            rank_dev = torch.zeros((w.Bt, w.Hkv, w.Blc), dtype=torch.int32, device="cuda")
+            B.dkv_ranks(c.h, l, rank_dev)
+            torch.cuda.synchronize()
+            rank_now = rank_dev.cpu().numpy()
             for b in range(w.Bt):
                 n = int(counts[b, l])
                 for h in range(w.Hkv):
