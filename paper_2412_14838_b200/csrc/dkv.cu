@@ -39,7 +39,8 @@ struct dkv_ctx {
   unsigned int* d_rb_hist2;   // [Bt][L][1024]
   int* d_status;        // [8]
   int sort_n;
-  size_t shrink_smem;
+  bool sel_reg;         // a head's scores fit the select kernel's registers and shared memory
+  size_t sel_smem;
   // tensor-core scoring
   int n_sms, tc_grid, tc_slots;
   float2* d_tc_stats;   // [3][Bt*Hkv][tc_slots][256]: partial softmax statistics, three layers in rotation
@@ -215,16 +216,15 @@ int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_
 }
 
 // ---- step (2): per-head top-Bl' ----------------------------------------------------------------
-int do_ranks(dkv_ctx* c, int layer, int* rank_out, cudaStream_t st) {
+int do_kept_sorted(dkv_ctx* c, int layer, int* sorted_out, cudaStream_t st) {
   const Shape& s = c->s;
-  rank_kernel<<<s.Bt * s.Hkv, kSelThreads, (size_t)c->sort_n * 8, st>>>(
-      c->d_scores + (size_t)layer * layer_scores(s), c->d_idx + (size_t)layer * layer_idx(s), c->d_held, rank_out,
-      s.P, s.Blc, c->sort_n, s.Hkv, s.L, layer);
+  kept_sorted_kernel<<<s.Bt * s.Hkv, kSelThreads, (size_t)((s.P + 31) / 32) * 4, st>>>(
+      c->d_idx + (size_t)layer * layer_idx(s), c->d_held, sorted_out, s.P, s.Blc, s.Hkv, s.L, layer);
   DKV_LAUNCHED(c);
   return DKV_OK;
 }
 
-int do_select(dkv_ctx* c, int layer, int* idx_out, cudaStream_t st) {
+int do_select(dkv_ctx* c, int layer, int* sorted_out, int* rank_out, cudaStream_t st) {
   const Shape& s = c->s;
   const size_t heads = (size_t)s.Bt * s.Hkv;
   ProfScope ps(c, DKV_STEP_SELECT, 1, st);
@@ -233,12 +233,12 @@ int do_select(dkv_ctx* c, int layer, int* idx_out, cudaStream_t st) {
   unsigned int* hh = c->d_head_hist + (size_t)layer * heads * kBins;
   unsigned int* ho = c->d_head_offs + (size_t)layer * heads * kBins;
   uint32_t* gr = c->d_grouped + (size_t)layer * layer_scores(s);
-  if ((s.P + kSelThreads - 1) / kSelThreads <= kRegChunk)
-    select_topk_kernel<true><<<(unsigned)heads, kSelThreads, 0, st>>>(sc, idx, idx_out, hh, ho, gr, s.P, s.Blc, c->d_count,
-                                                                     s.Hkv, s.L, layer);
+  if (c->sel_reg)
+    select_topk_kernel<true><<<(unsigned)heads, kSelThreads, c->sel_smem, st>>>(
+        sc, idx, sorted_out, rank_out, hh, ho, gr, s.P, s.Blc, c->sort_n, c->d_count, s.Hkv, s.L, layer);
   else
-    select_topk_kernel<false><<<(unsigned)heads, kSelThreads, 0, st>>>(sc, idx, idx_out, hh, ho, gr, s.P, s.Blc, c->d_count,
-                                                                      s.Hkv, s.L, layer);
+    select_topk_kernel<false><<<(unsigned)heads, kSelThreads, c->sel_smem, st>>>(
+        sc, idx, sorted_out, rank_out, hh, ho, gr, s.P, s.Blc, c->sort_n, c->d_count, s.Hkv, s.L, layer);
   DKV_LAUNCHED(c);
   c->selected[layer] = 1;
   c->gathered[layer] = c->stale[layer] = 0;
@@ -277,9 +277,8 @@ int do_shrink(dkv_ctx* c, int layer0, int n, void* const* kb, void* const* vb, c
   LayerPtrs ptrs;
   for (int i = 0; i < n; ++i) { ptrs.kb[layer0 + i] = kb[i]; ptrs.vb[layer0 + i] = vb[i]; }
   ProfScope ps(c, DKV_STEP_SHRINK, 2, st);
-  shrink_kernel<<<dim3(s.Bt * s.Hkv, n), kShrinkThreads, c->shrink_smem, st>>>(
-      ptrs, layer0, c->d_scores, c->d_idx, c->d_count, c->d_held, s.Bt, s.Hkv, s.L, s.P, s.ws, s.Blc, s.rows,
-      s.D * 2 / 16, layer_idx(s), layer_scores(s));
+  shrink_kernel<<<dim3(s.Bt * s.Hkv, n, 2), kShrinkThreads, 0, st>>>(ptrs, layer0, c->d_count, c->d_held, s.Hkv, s.L, s.ws,
+                                                                      s.rows, s.D * 2 / 16);
   DKV_LAUNCHED(c);
   commit_held_kernel<<<(s.Bt * n + 127) / 128, 128, 0, st>>>(c->d_held, c->d_count, s.Bt, s.L, layer0, n);
   DKV_LAUNCHED(c);
@@ -339,7 +338,7 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
     c->scored[el] = 1;
     DKV_CUDA(c, cudaEventRecord(c->ev_scored[el], st));
     DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_scored[el], 0));
-    if ((rc = do_select(c, el, nullptr, sd))) return rc;
+    if ((rc = do_select(c, el, nullptr, nullptr, sd))) return rc;
     if ((rc = do_gather(c, el, k[el], v[el], kb[el], vb[el], sd))) return rc;
     const bool update = ((el + 1) % s.m == 0) || (el + 1 == s.L && s.L % s.m != 0);
     if (update) {
@@ -482,9 +481,14 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMemset(c->d_count, 0, sizeof(int) * bl));
   TRY(cudaMemset(c->d_held, 0, sizeof(int) * bl));
   TRY(cudaMemset(c->d_dbg, 0, sizeof(int) * 3 * bl));
-  c->shrink_smem = sizeof(int) * (size_t)(s.Blc > kBins ? s.Blc : kBins);
-  TRY(cudaFuncSetAttribute(rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, c->sort_n * 8));
-  TRY(cudaFuncSetAttribute(shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->shrink_smem));
+  {
+    c->sel_reg = (s.P + kSelThreads - 1) / kSelThreads <= kRegChunk;
+    size_t stage = (size_t)c->sort_n * 8;
+    if (c->sel_reg && (size_t)s.P * 4 > stage) stage = (size_t)s.P * 4;
+    c->sel_smem = ((stage + 15) & ~(size_t)15) + (size_t)s.Blc * 4;
+  }
+  TRY(cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem));
+  TRY(cudaFuncSetAttribute(select_topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem));
 #undef TRY
   if (e != cudaSuccess) {
     rc = e == cudaErrorMemoryAllocation ? DKV_ERR_NOMEM : DKV_ERR_CUDA;
@@ -533,15 +537,7 @@ int dkv_select_topk(dkv_ctx* c, int32_t layer, int32_t* idx_out, int32_t* rank_o
   int rc = check_layer(c, layer);
   if (rc) return rc;
   if (!c->scored[layer]) return DKV_ERR_STATE;
-  rc = do_select(c, layer, idx_out, as_stream(stream));
-  if (rc || !rank_out) return rc;
-  // ranks of a fresh selection: every head holds Bl' positions
-  const Shape& s = c->s;
-  rank_kernel<<<s.Bt * s.Hkv, kSelThreads, (size_t)c->sort_n * 8, as_stream(stream)>>>(
-      c->d_scores + (size_t)layer * layer_scores(s), c->d_idx + (size_t)layer * layer_idx(s), c->d_count, rank_out,
-      s.P, s.Blc, c->sort_n, s.Hkv, s.L, layer);
-  DKV_LAUNCHED(c);
-  return DKV_OK;
+  return do_select(c, layer, idx_out, rank_out, as_stream(stream));
 }
 
 int dkv_rebudget(dkv_ctx* c, int32_t upto_layer, int32_t* counts_out, void* stream) {
@@ -613,7 +609,7 @@ int dkv_run_prefill_pass_host(dkv_ctx* c, const void* const* q_win, const void* 
     DKV_CUDA(c, cudaEventRecord(c->ev_copied[slot], cp));
     DKV_CUDA(c, cudaStreamWaitEvent(st, c->ev_copied[slot], 0));
     if ((rc = do_score(c, l, c->st_q[slot], c->st_k[slot], nullptr, st))) return rc;
-    if ((rc = do_select(c, l, nullptr, st))) return rc;
+    if ((rc = do_select(c, l, nullptr, nullptr, st))) return rc;
     if ((rc = do_gather(c, l, c->st_k[slot], c->st_v[slot], c->st_kb[l], c->st_vb[l], st))) return rc;
     DKV_CUDA(c, cudaEventRecord(c->ev_consumed[slot], st));
     const bool update = ((l + 1) % s.m == 0) || (l + 1 == s.L && s.L % s.m != 0);
@@ -649,12 +645,12 @@ int dkv_layer_views(dkv_ctx* c, int32_t layer, const float** scores, const int32
   return DKV_OK;
 }
 
-int dkv_ranks(dkv_ctx* c, int32_t layer, int32_t* rank_out, void* stream) {
+int dkv_kept_sorted(dkv_ctx* c, int32_t layer, int32_t* sorted_out, void* stream) {
   int rc = check_layer(c, layer);
   if (rc) return rc;
-  if (!rank_out) return DKV_ERR_INVALID_ARG;
+  if (!sorted_out) return DKV_ERR_INVALID_ARG;
   if (!c->gathered[layer]) return DKV_ERR_STATE;
-  return do_ranks(c, layer, rank_out, as_stream(stream));
+  return do_kept_sorted(c, layer, sorted_out, as_stream(stream));
 }
 
 int dkv_budget_views(dkv_ctx* c, const int32_t** cnt, const int32_t** z, const int32_t** zp, const int32_t** held) {

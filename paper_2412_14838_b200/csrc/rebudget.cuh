@@ -37,14 +37,22 @@ rb_locate_kernel(const unsigned int* __restrict__ head_hist, const unsigned int*
   __shared__ int sm_scan[33];
   __shared__ int found[2];
   const int b = blockIdx.x, tid = threadIdx.x;
-  for (int bin = tid; bin < kBins; bin += 1024) {
-    unsigned int s = 0;
-    for (int ih = 0; ih < l * Hkv; ++ih) {
+  for (int bin = tid; bin < kBins; bin += 1024) { hist[bin] = 0; hist1[(size_t)b * kBins + bin] = 0; }
+  __syncthreads();
+  {
+    // four groups of 256 threads walk the (layer, head) list in parallel, eight digits per thread
+    const int g = tid >> 8, c = tid & 255;
+    uint4 a0 = make_uint4(0, 0, 0, 0), a1 = make_uint4(0, 0, 0, 0);
+    for (int ih = g; ih < l * Hkv; ih += 4) {
       const int i = ih / Hkv, h = ih % Hkv;
-      s += head_hist[(((size_t)i * Bt + b) * Hkv + h) * kBins + bin];
+      const uint4* src = reinterpret_cast<const uint4*>(head_hist + (((size_t)i * Bt + b) * Hkv + h) * kBins) + 2 * c;
+      const uint4 x = src[0], y = src[1];
+      a0.x += x.x; a0.y += x.y; a0.z += x.z; a0.w += x.w;
+      a1.x += y.x; a1.y += y.y; a1.z += y.z; a1.w += y.w;
     }
-    hist[bin] = s;
-    hist1[(size_t)b * kBins + bin] = 0;
+    unsigned int* hb = hist + 8 * c;
+    atomicAdd(hb + 0, a0.x); atomicAdd(hb + 1, a0.y); atomicAdd(hb + 2, a0.z); atomicAdd(hb + 3, a0.w);
+    atomicAdd(hb + 4, a1.x); atomicAdd(hb + 5, a1.y); atomicAdd(hb + 6, a1.z); atomicAdd(hb + 7, a1.w);
   }
   for (int e = tid; e < L; e += 1024) above2[b * L + e] = 0;
   for (int e = tid; e < l * 1024; e += 1024) hist2[(size_t)b * L * 1024 + e] = 0;

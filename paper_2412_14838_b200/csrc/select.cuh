@@ -5,6 +5,9 @@
 // Scores are non-negative floats, so their bit patterns order like unsigned integers.  The
 // threshold T (bit pattern of the B^l-th largest score) is found by a 3-pass radix select,
 // most significant digit first (11 + 11 + 10 bits), with a shared-memory histogram per pass.
+// The kept positions are then compacted in position order and sorted by (score descending,
+// position ascending): that is the order Algorithm 1's topk() returns and stores them in, and a
+// later truncation to a smaller budget is a prefix of it.
 // The first pass's histogram (top 11 bits: sign, exponent, 2 mantissa bits) is also kept per head
 // in global memory, together with a copy of the head's scores grouped by that digit, so that
 // Update_Buffer_Length can locate the global K-th value from histograms and then look only at
@@ -16,7 +19,7 @@ namespace dkv {
 
 constexpr int kSelThreads = 1024;
 constexpr int kBins = 2048;               // 11-bit digits
-constexpr int kRegChunk = 32;             // positions per thread held in registers
+constexpr int kRegChunk = 32;             // scores per thread held in registers
 
 __device__ __forceinline__ int digit_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
 __device__ __forceinline__ uint32_t digit_mask(int pass) { return pass == 2 ? 1023u : 2047u; }
@@ -69,30 +72,77 @@ __device__ __forceinline__ void find_digit(const unsigned int* hist, int nbins, 
   __syncthreads();
 }
 
-// scores: [Bt*Hkv][P] of one layer.  idx: [Bt*Hkv][keep] kept positions, ascending.
+// Warp-aggregated counter bump: lanes with equal `digit` share one atomicAdd.  Inactive lanes pass
+// active = false.  Returns, for active lanes, a distinct slot: old counter value + rank inside the group.
+// Must be called by all 32 lanes.
+__device__ __forceinline__ unsigned int agg_bump(unsigned int* counters, unsigned int digit, bool active) {
+  const unsigned int lane = threadIdx.x & 31;
+  const unsigned int key = active ? digit : 0xFFFFFFFFu;
+  const unsigned int peers = __match_any_sync(0xFFFFFFFFu, key);
+  const int leader = __ffs(peers) - 1;
+  unsigned int base = 0;
+  if (active && (int)lane == leader) base = atomicAdd(&counters[digit], (unsigned int)__popc(peers));
+  base = __shfl_sync(0xFFFFFFFFu, base, leader);
+  return base + (unsigned int)__popc(peers & ((1u << lane) - 1u));
+}
+
+// Bitonic sort of keys[0 .. sort_n) ascending; sort_n a power of two.  Ends with a barrier.
+__device__ __forceinline__ void bitonic_sort(unsigned long long* keys, int sort_n) {
+  for (int size = 2; size <= sort_n; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int t = threadIdx.x; t < (sort_n >> 1); t += blockDim.x) {
+        const int lo = ((t / stride) * stride * 2) + (t % stride);
+        const int hi = lo + stride;
+        const bool up = ((lo & size) == 0);
+        const unsigned long long a = keys[lo], b = keys[hi];
+        if ((a > b) == up) { keys[lo] = b; keys[hi] = a; }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// scores: [Bt*Hkv][P] of one layer.
+// idx: [Bt*Hkv][keep] kept positions in buffer order = (score descending, position ascending).
+// sorted_out (optional): the same positions ascending; rank_out (optional): rank of each of those.
 // head_hist, head_offs: [Bt*Hkv][2048] first-digit counts of the head and their ascending exclusive offsets.
 // grouped: [Bt*Hkv][P] the head's score bits grouped by first digit (ascending digit; order inside a
 // group is unspecified).  Also records count[b][layer] = keep.
+// Every warp owns a run of 32*chunk consecutive positions; lane j holds positions run + 32*e + j.
+// Dynamic shared memory: max(REG ? 4*P : 0, 8*sort_n) bytes rounded up to 16, then 4*keep bytes.
 template <bool REG>
 __global__ void __launch_bounds__(kSelThreads)
-select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int* __restrict__ idx_out,
-                   unsigned int* __restrict__ head_hist, unsigned int* __restrict__ head_offs,
-                   uint32_t* __restrict__ grouped, int P, int keep, int* __restrict__ count, int Hkv, int L, int layer) {
+select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int* __restrict__ sorted_out,
+                   int* __restrict__ rank_out, unsigned int* __restrict__ head_hist, unsigned int* __restrict__ head_offs,
+                   uint32_t* __restrict__ grouped, int P, int keep, int sort_n, int* __restrict__ count, int Hkv, int L,
+                   int layer) {
+  extern __shared__ __align__(16) unsigned char dyn[];
   __shared__ unsigned int hist[kBins];
   __shared__ int sm_scan[33], sm_scan2[33];
   __shared__ int found[2];
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t* v = reinterpret_cast<const uint32_t*>(scores) + (size_t)blockIdx.x * P;
   if (tid == 0 && blockIdx.x % Hkv == 0) count[(blockIdx.x / Hkv) * L + layer] = keep;
 
+  const size_t stage_bytes = ((REG ? (size_t)P * 4 : 0) > (size_t)sort_n * 8 ? (size_t)P * 4 : (size_t)sort_n * 8);
+  uint32_t* stage = reinterpret_cast<uint32_t*>(dyn);                       // grouped scores (REG), later sort keys
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(dyn);
+  int* sel_pos = reinterpret_cast<int*>(dyn + ((stage_bytes + 15) & ~(size_t)15));
+
   const int chunk = (P + kSelThreads - 1) / kSelThreads;       // REG: chunk <= kRegChunk
-  const int p0 = min(P, tid * chunk), p1 = min(P, p0 + chunk);
-  const int n_mine = p1 - p0;
+  const int run0 = warp * chunk * 32;
+  const int n_e = REG ? kRegChunk : chunk;
   uint32_t r[REG ? kRegChunk : 1];
-  if (REG) {
+  if constexpr (REG) {
 #pragma unroll
-    for (int e = 0; e < kRegChunk; ++e) r[e] = (e < n_mine) ? v[p0 + e] : 0u;
+    for (int e = 0; e < kRegChunk; ++e) { const int p = run0 + e * 32 + lane; r[e] = (e < chunk && p < P) ? v[p] : 0u; }
   }
+#define DKV_SEL_FOR(e) _Pragma("unroll") for (int e = 0; e < n_e; ++e)
+#define DKV_SEL_POS(e) (run0 + (e) * 32 + lane)
+#define DKV_SEL_OK(e) ((e) < chunk && DKV_SEL_POS(e) < P)
+  auto val = [&](int e) -> uint32_t {
+    if constexpr (REG) return r[e]; else return DKV_SEL_OK(e) ? v[DKV_SEL_POS(e)] : 0u;
+  };
 
   uint32_t prefix = 0, mask = 0;
   int need = keep, total = P;
@@ -101,12 +151,11 @@ select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int*
     const uint32_t dm = digit_mask(pass);
     for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
     __syncthreads();
-    if (REG) {
-#pragma unroll
-      for (int e = 0; e < kRegChunk; ++e)
-        if (e < n_mine && (r[e] & mask) == prefix) atomicAdd(&hist[(r[e] >> shift) & dm], 1u);
-    } else {
-      for (int e = 0; e < n_mine; ++e) { const uint32_t u = v[p0 + e]; if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & dm], 1u); }
+    DKV_SEL_FOR(e) {
+      const uint32_t u = val(e);
+      const bool in = DKV_SEL_OK(e) && (u & mask) == prefix;
+      if (pass == 0) agg_bump(hist, (u >> shift) & dm, in);          // neighbours share digits after pooling
+      else if (in) atomicAdd(&hist[(u >> shift) & dm], 1u);
     }
     __syncthreads();
     if (pass == 0) {
@@ -123,12 +172,15 @@ select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int*
       for (int i = tid; i < kBins; i += kSelThreads) hist[i] = go[i];
       __syncthreads();
       uint32_t* dst = grouped + (size_t)blockIdx.x * P;
-      if (REG) {
-#pragma unroll
-        for (int e = 0; e < kRegChunk; ++e)
-          if (e < n_mine) dst[atomicAdd(&hist[r[e] >> 21], 1u)] = r[e];
-      } else {
-        for (int e = 0; e < n_mine; ++e) { const uint32_t u = v[p0 + e]; dst[atomicAdd(&hist[u >> 21], 1u)] = u; }
+      DKV_SEL_FOR(e) {
+        const uint32_t u = val(e);
+        const bool in = DKV_SEL_OK(e);
+        const unsigned int slot = agg_bump(hist, u >> 21, in);
+        if (in) { if constexpr (REG) stage[slot] = u; else dst[slot] = u; }
+      }
+      if constexpr (REG) {
+        __syncthreads();
+        for (int i = tid; i < P; i += kSelThreads) dst[i] = stage[i];
       }
     }
     total = cnt_d;
@@ -140,75 +192,73 @@ select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int*
   const uint32_t T = prefix;
   const int need_eq = need;                 // how many of the entries equal to T are kept (lowest positions)
 
-  // Ordered compaction: each thread owns a contiguous run of positions.
+  // Ordered compaction.  Position order inside a warp's run is (e, lane), so ballots give the order.
   int gt = 0, eq = 0;
-  if (REG) {
+  DKV_SEL_FOR(e) { const uint32_t u = val(e); if (DKV_SEL_OK(e)) { gt += (u > T); eq += (u == T); } }
 #pragma unroll
-    for (int e = 0; e < kRegChunk; ++e) if (e < n_mine) { gt += (r[e] > T); eq += (r[e] == T); }
-  } else {
-    for (int e = 0; e < n_mine; ++e) { const uint32_t u = v[p0 + e]; gt += (u > T); eq += (u == T); }
-  }
+  for (int o = 16; o > 0; o >>= 1) { gt += __shfl_xor_sync(0xFFFFFFFFu, gt, o); eq += __shfl_xor_sync(0xFFFFFFFFu, eq, o); }
   int tot_gt, tot_eq;
-  int g = block_excl_scan(gt, sm_scan, &tot_gt);
-  int q = block_excl_scan(eq, sm_scan2, &tot_eq);
-  int* my_idx = idx + (size_t)blockIdx.x * keep;
-  int* my_out = idx_out ? idx_out + (size_t)blockIdx.x * keep : nullptr;
-  if (REG) {
-#pragma unroll
-    for (int e = 0; e < kRegChunk; ++e) {
-      if (e < n_mine) {
-        const uint32_t u = r[e];
-        const bool is_eq = (u == T);
-        if (u > T || (is_eq && q < need_eq)) {
-          const int out = g + min(q, need_eq);
-          my_idx[out] = p0 + e;
-          if (my_out) my_out[out] = p0 + e;
-        }
-        g += (u > T); q += is_eq;
-      }
+  int g_run = block_excl_scan(lane == 0 ? gt : 0, sm_scan, &tot_gt);       // one value per warp, carried by lane 0
+  int q_run = block_excl_scan(lane == 0 ? eq : 0, sm_scan2, &tot_eq);
+  g_run = __shfl_sync(0xFFFFFFFFu, g_run, 0);
+  q_run = __shfl_sync(0xFFFFFFFFu, q_run, 0);
+  const unsigned int lt = (1u << lane) - 1u;
+  int* my_sorted = sorted_out ? sorted_out + (size_t)blockIdx.x * keep : nullptr;
+  DKV_SEL_FOR(e) {
+    const uint32_t u = val(e);
+    const bool ok = DKV_SEL_OK(e);
+    const bool is_gt = ok && u > T, is_eq = ok && u == T;
+    const unsigned int bg = __ballot_sync(0xFFFFFFFFu, is_gt), be = __ballot_sync(0xFFFFFFFFu, is_eq);
+    const int g = g_run + __popc(bg & lt), q = q_run + __popc(be & lt);
+    if (is_gt || (is_eq && q < need_eq)) {
+      const int out = g + min(q, need_eq);
+      const int p = DKV_SEL_POS(e);
+      sel_pos[out] = p;
+      if (my_sorted) my_sorted[out] = p;
+      keys[out] = ((unsigned long long)(~u) << 32) | (unsigned int)out;
     }
-  } else {
-    for (int e = 0; e < n_mine; ++e) {
-      const uint32_t u = v[p0 + e];
-      const bool is_eq = (u == T);
-      if (u > T || (is_eq && q < need_eq)) {
-        const int out = g + min(q, need_eq);
-        my_idx[out] = p0 + e;
-        if (my_out) my_out[out] = p0 + e;
-      }
-      g += (u > T); q += is_eq;
-    }
+    g_run += __popc(bg); q_run += __popc(be);
   }
+  for (int i = tid + keep; i < sort_n; i += kSelThreads) keys[i] = ~0ull;
+  __syncthreads();
+  bitonic_sort(keys, sort_n);
+  int* my_idx = idx + (size_t)blockIdx.x * keep;
+  for (int i = tid; i < keep; i += kSelThreads) {
+    const int slot = (int)(keys[i] & 0xFFFFFFFFull);
+    my_idx[i] = sel_pos[slot];
+    if (rank_out) rank_out[(size_t)blockIdx.x * keep + slot] = i;
+  }
+#undef DKV_SEL_FOR
+#undef DKV_SEL_POS
+#undef DKV_SEL_OK
 }
 
-// Rank of every held position among the held positions of its head, in (score descending, position
-// ascending) order; equals its rank among all positions, because the held set is a top-n of that order.
-// One CTA per (sample, head); dynamic shared memory = sort_n * 8 bytes, sort_n = power of two >= idx_stride.
+// Ascending list of the positions a head currently holds: sorted_out[b,h,0:held] (one CTA per head).
+// Dynamic shared memory: ceil(P / 32) words (one bit per position).
 __global__ void __launch_bounds__(kSelThreads)
-rank_kernel(const float* __restrict__ scores, const int* __restrict__ idx, const int* __restrict__ held,
-            int* __restrict__ rank_out, int P, int idx_stride, int sort_n, int Hkv, int L, int layer) {
-  extern __shared__ __align__(16) unsigned long long skeys[];
+kept_sorted_kernel(const int* __restrict__ idx, const int* __restrict__ held, int* __restrict__ sorted_out, int P,
+                   int idx_stride, int Hkv, int L, int layer) {
+  extern __shared__ unsigned int bits[];
+  __shared__ int sm_scan[33];
   const int tid = threadIdx.x;
   const int n = held[(blockIdx.x / Hkv) * L + layer];
-  const uint32_t* v = reinterpret_cast<const uint32_t*>(scores) + (size_t)blockIdx.x * P;
-  const int* my_idx = idx + (size_t)blockIdx.x * idx_stride;
-  for (int i = tid; i < sort_n; i += kSelThreads)
-    skeys[i] = i < n ? (((unsigned long long)(~v[my_idx[i]]) << 32) | (unsigned int)i) : ~0ull;
+  const int words = (P + 31) / 32;
+  for (int i = tid; i < words; i += kSelThreads) bits[i] = 0;
   __syncthreads();
-  for (int size = 2; size <= sort_n; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      for (int t = tid; t < (sort_n >> 1); t += kSelThreads) {
-        const int lo = ((t / stride) * stride * 2) + (t % stride);
-        const int hi = lo + stride;
-        const bool up = ((lo & size) == 0);
-        const unsigned long long a = skeys[lo], b = skeys[hi];
-        if ((a > b) == up) { skeys[lo] = b; skeys[hi] = a; }
-      }
-      __syncthreads();
-    }
+  const int* my = idx + (size_t)blockIdx.x * idx_stride;
+  for (int i = tid; i < n; i += kSelThreads) { const int p = my[i]; atomicOr(&bits[p >> 5], 1u << (p & 31)); }
+  __syncthreads();
+  const int per = (words + kSelThreads - 1) / kSelThreads;
+  const int w0 = min(words, tid * per), w1 = min(words, w0 + per);
+  int mine = 0;
+  for (int w = w0; w < w1; ++w) mine += __popc(bits[w]);
+  int tot;
+  int out = block_excl_scan(mine, sm_scan, &tot);
+  int* dst = sorted_out + (size_t)blockIdx.x * idx_stride;
+  for (int w = w0; w < w1; ++w) {
+    unsigned int m = bits[w];
+    while (m) { const int b = __ffs(m) - 1; dst[out++] = w * 32 + b; m &= m - 1; }
   }
-  for (int i = tid; i < n; i += kSelThreads)
-    rank_out[(size_t)blockIdx.x * idx_stride + (int)(skeys[i] & 0xFFFFFFFFull)] = i;
 }
 
 }  // namespace dkv
