@@ -117,9 +117,11 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
 int dkv_set_scores(dkv_ctx* ctx, int32_t layer, const float* scores, void* stream);
 
 /* (2) Eq. 3 / Algorithm 1 "topk(B^l)".  Per (b, h): the Bl' positions with the largest score under the
- *     total order (score descending, position ascending).
- *     idx_out  : int32 [Bt, Hkv, Bl'] kept positions, ascending (optional)
- *     rank_out : int32 [Bt, Hkv, Bl'] place of each kept position in the total order, 0 = best (optional)
+ *     total order (score descending, position ascending).  The context keeps them in that order, which
+ *     is the order Algorithm 1's topk() yields and the order of the buffer rows dkv_compact writes.
+ *     idx_out  : int32 [Bt, Hkv, Bl'] the kept positions, ascending (optional)
+ *     rank_out : int32 [Bt, Hkv, Bl'] place of each of those in the total order, 0 = best, i.e. its
+ *                buffer row (optional)
  *     Sets count[b][layer] = Bl'.  Needs the layer's scores (else DKV_ERR_STATE).  Also files the head's
  *     scores by their leading bits for the later global top-K of dkv_rebudget. */
 int dkv_select_topk(dkv_ctx* ctx, int32_t layer, int32_t* idx_out, int32_t* rank_out, void* stream);
@@ -131,15 +133,15 @@ int dkv_select_topk(dkv_ctx* ctx, int32_t layer, int32_t* idx_out, int32_t* rank
  *     counts_out : int32 [Bt, L] device copy of the counts after the update (optional). */
 int dkv_rebudget(dkv_ctx* ctx, int32_t upto_layer, int32_t* counts_out, void* stream);
 
-/* (4) Algorithm 1's buffer build and truncation for one layer.
- *     k_src, v_src != NULL : gather.  kb[b,h,0:c] = k_src[b,h,idx[0:c]], kb[b,h,c:c+ws] = k_src[b,h,P:S],
+/* (4) Algorithm 1's buffer build and truncation for one layer.  Buffer rows are in Algorithm 1's own
+ *     order: row r of a head holds its r-th best position (score descending, ties by position), so
+ *     that truncating to a smaller count keeps a prefix; the ws window rows follow the kept rows.
+ *     k_src, v_src != NULL : gather.  kb[b,h,r] = k_src[b,h,pos_r] for r < c, kb[b,h,c:c+ws] = k_src[b,h,P:S],
  *                            same for v; c = count[b][layer].  k_src, v_src : bf16 [Bt, Hkv, S, D].
- *     k_src == v_src == NULL : shrink kb/vb in place to the current count: the count[b][layer] best of the
- *                            held rows (score descending, position ascending) stay, in position order,
- *                            followed by the ws window rows.
+ *     k_src == v_src == NULL : shrink kb/vb in place to the current count c: rows [0, c) stay, the window
+ *                            rows move up behind them.
  *     kb, vb  : bf16 [Bt, Hkv, Bl' + ws, D] fixed stride; rows past the valid length are unspecified.
- *     len_out : int32 [Bt, Hkv] valid rows including the window (optional).
- *     The context's kept positions are compacted with the rows. */
+ *     len_out : int32 [Bt, Hkv] valid rows including the window (optional). */
 int dkv_compact(dkv_ctx* ctx, int32_t layer, const void* k_src, const void* v_src, void* kb, void* vb,
                 int32_t* len_out, void* stream);
 
@@ -163,13 +165,13 @@ int dkv_run_prefill_pass_host(dkv_ctx* ctx, const void* const* q_win, const void
 /* Copy the current counts to host int32 [Bt, L] (synchronises `stream`). */
 int dkv_get_counts(dkv_ctx* ctx, int32_t* host_counts, void* stream);
 /* Device-side views for inspection, owned by the context: the history scores of a layer
- * (fp32 [Bt,Hkv,P]) and its current kept positions (int32 [Bt,Hkv,Bl'], the first held[b][layer]
- * entries of each head valid).  Either out pointer may be NULL. */
+ * (fp32 [Bt,Hkv,P]) and the positions it currently keeps, in buffer order (int32 [Bt,Hkv,Bl'], the
+ * first held[b][layer] entries of each head valid; entry r is the position of buffer row r).
+ * Either out pointer may be NULL. */
 int dkv_layer_views(dkv_ctx* ctx, int32_t layer, const float** scores, const int32_t** idx);
-/* Rank (place in the order score descending, position ascending; 0 = best) of every position a gathered
- * layer currently holds: rank_out int32 [Bt,Hkv,Bl'], device, first held[b][layer] entries per head
- * written.  This is the order Algorithm 1 stores its buffers in; the buffers here are in position order. */
-int dkv_ranks(dkv_ctx* ctx, int32_t layer, int32_t* rank_out, void* stream);
+/* The positions a gathered layer currently keeps, ascending: sorted_out int32 [Bt,Hkv,Bl'], device,
+ * the first held[b][layer] entries of each head written. */
+int dkv_kept_sorted(dkv_ctx* ctx, int32_t layer, int32_t* sorted_out, void* stream);
 /* Device-side views of the last update's intermediate integers, int32 [Bt, L] each:
  * cnt (Eq. 4 hits per layer), Z (Eq. 5), Zp (Eq. 6), and held (rows each layer's buffers hold now). */
 int dkv_budget_views(dkv_ctx* ctx, const int32_t** cnt, const int32_t** z, const int32_t** zp, const int32_t** held);

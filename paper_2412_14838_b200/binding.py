@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(HERE, "libdkv.so")
 EXPORTS = [
     "dkv_create", "dkv_destroy", "dkv_reset", "dkv_score", "dkv_score_static", "dkv_set_scores", "dkv_select_topk", "dkv_rebudget",
     "dkv_compact", "dkv_compact_all", "dkv_run_prefill_pass", "dkv_run_prefill_pass_host", "dkv_get_counts",
-    "dkv_layer_views", "dkv_ranks", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status", "dkv_profile", "dkv_profile_read", "dkv_launch_count", "dkv_last_cuda_error",
+    "dkv_layer_views", "dkv_kept_sorted", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status", "dkv_profile", "dkv_profile_read", "dkv_launch_count", "dkv_last_cuda_error",
     "dkv_strerror", "dkv_version",
 ]
 
@@ -64,7 +64,7 @@ def load() -> ctypes.CDLL:
         "dkv_run_prefill_pass_host": [vp, pp, pp, pp, pp, pp, vp],
         "dkv_get_counts": [vp, vp, vp],
         "dkv_layer_views": [vp, i32, pp, pp],
-        "dkv_ranks": [vp, i32, vp, vp],
+        "dkv_kept_sorted": [vp, i32, vp, vp],
         "dkv_budget_views": [vp, pp, pp, pp, pp],
         "dkv_memcpy_to_host": [vp, vp, vp, ctypes.c_uint64, vp],
         "dkv_last_status": [vp, vp],
@@ -200,14 +200,14 @@ def dkv_get_counts(ctx: int, host_counts, stream=None) -> None:
 
 
 def dkv_layer_views(ctx: int, layer: int):
-    """Device addresses (scores, idx) of one layer's state inside the context."""
+    """Device addresses (scores, kept positions in buffer order) of one layer's state inside the context."""
     a, b = ctypes.c_void_p(), ctypes.c_void_p()
     _check(load().dkv_layer_views(ctx, layer, ctypes.byref(a), ctypes.byref(b)), "dkv_layer_views")
     return a.value, b.value
 
 
-def dkv_ranks(ctx: int, layer: int, rank_out, stream=None) -> None:
-    _check(load().dkv_ranks(ctx, layer, _ptr(rank_out), _stream(stream)), "dkv_ranks")
+def dkv_kept_sorted(ctx: int, layer: int, sorted_out, stream=None) -> None:
+    _check(load().dkv_kept_sorted(ctx, layer, _ptr(sorted_out), _stream(stream)), "dkv_kept_sorted")
 
 
 def dkv_budget_views(ctx: int):

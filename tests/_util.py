@@ -60,3 +60,10 @@ def global_cut_gap(history, k):
     lo = part[flat.size - k - 1]
     hi = part[flat.size - k:].min()
     return (hi - lo) / hi if hi > 0 else 0.0
+
+
+def buffer_order(rows: np.ndarray, rank: np.ndarray, n: int) -> np.ndarray:
+    """Oracle rows (kept rows in position order, then window rows) rearranged into the library's buffer
+    order: kept rows by rank (score descending, ties by position), window rows last."""
+    order = np.argsort(np.asarray(rank[:n]), kind="stable")
+    return np.concatenate([rows[:n][order], rows[n:]], axis=0)

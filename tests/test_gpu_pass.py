@@ -63,13 +63,14 @@ class GpuPass:
         B.dkv_memcpy_to_host(self.h, out, B.dkv_layer_views(self.h, layer)[0], out.nbytes)
         return out
 
-    def idx_rank(self, layer):
+    def kept(self, layer):
+        """(positions ascending, positions in buffer order), int32 [Bt,Hkv,Blc] each."""
         w = self.w
         _, ia = B.dkv_layer_views(self.h, layer)
-        rank = torch.zeros((w.Bt, w.Hkv, w.Blc), dtype=torch.int32, device="cuda")
-        B.dkv_ranks(self.h, layer, rank)
+        srt = torch.zeros((w.Bt, w.Hkv, w.Blc), dtype=torch.int32, device="cuda")
+        B.dkv_kept_sorted(self.h, layer, srt)
         torch.cuda.synchronize()
-        return B.read_device_i32(self.h, ia, (w.Bt, w.Hkv, w.Blc)), rank.cpu().numpy()
+        return srt.cpu().numpy(), B.read_device_i32(self.h, ia, (w.Bt, w.Hkv, w.Blc))
 
     def close(self):
         B.dkv_destroy(self.h)
@@ -82,27 +83,27 @@ def check_properties(g: GpuPass):
     assert (g.counts >= 0).all() and (g.counts <= w.Blc).all()
     assert (g.counts.sum(axis=1) <= w.N * w.L).all(), "global budget exceeded"
     for l in range(w.L):
-        idx, rank = g.idx_rank(l)
+        srt, buf_idx = g.kept(l)
         sc = torch.from_numpy(g.scores(l)).cuda()
         for b in range(w.Bt):
             n = int(g.counts[b, l])
-            ii = torch.from_numpy(idx[b, :, :n].astype(np.int64)).cuda()           # [Hkv, n]
-            rr = rank[b, :, :n]
-            assert (np.diff(idx[b, :, :n], axis=1) > 0).all() and (idx[b, :, :n] < w.P).all()
-            assert (np.sort(rr, axis=1) == np.arange(n)[None, :]).all(), "ranks are not 0..n-1"
+            assert (np.diff(srt[b, :, :n], axis=1) > 0).all() and (srt[b, :, :n] < w.P).all()
+            assert (np.sort(buf_idx[b, :, :n], axis=1) == srt[b, :, :n]).all(), "buffer order is not a permutation of the kept set"
+            ii = torch.from_numpy(buf_idx[b, :, :n].astype(np.int64)).cuda()       # [Hkv, n], buffer order
             # kept rows and window rows are byte copies of the layer's K/V
             for src, buf in ((g.k[l], g.kb[l]), (g.v[l], g.vb[l])):
                 want = torch.gather(src[b], 1, ii[:, :, None].expand(-1, -1, w.D))
                 assert torch.equal(buf[b, :, :n], want)
                 assert torch.equal(buf[b, :, n:n + w.ws], src[b, :, w.P:])
-            # every kept score >= every dropped score (per head), order by rank is non-increasing
+            # every kept score >= every dropped score (per head); buffer order = score descending, ties by position
             kept = torch.gather(sc[b], 1, ii)
             mask = torch.ones_like(sc[b], dtype=torch.bool).scatter_(1, ii, False)
             dropped_max = torch.where(mask, sc[b], torch.full_like(sc[b], -1.0)).max(dim=1).values
             if n:
                 assert (kept.min(dim=1).values >= dropped_max).all()
-                by_rank = torch.gather(kept, 1, torch.from_numpy(np.argsort(rr, axis=1)).cuda())
-                assert (by_rank[:, 1:] <= by_rank[:, :-1]).all()
+                assert (kept[:, 1:] <= kept[:, :-1]).all()
+                tie = kept[:, 1:] == kept[:, :-1]
+                assert (ii[:, 1:][tie] > ii[:, :-1][tie]).all(), "ties are not in position order"
 
 
 def compare_full(g: GpuPass, verbose_name=""):
@@ -126,7 +127,7 @@ def compare_full(g: GpuPass, verbose_name=""):
         assert min(gaps) <= U.NEAR_TIE, f"counts differ ({g.counts} vs {ref['counts']}) without a global near-tie"
         near += 1
     for l in range(w.L):
-        idx, _ = g.idx_rank(l)
+        idx, _ = g.kept(l)
         kb = g.kb[l].cpu().numpy().view(np.uint16)
         vb = g.vb[l].cpu().numpy().view(np.uint16)
         for b in range(w.Bt):
@@ -135,8 +136,9 @@ def compare_full(g: GpuPass, verbose_name=""):
                 exact, ev = U.select_matches(ref["score"][l][b, h], idx[b, h, :n], n)
                 near += ev
                 if exact and counts_equal:
-                    assert (kb[b, h, :n + w.ws] == ref["kb"][l][b][h]).all(), f"K bytes differ l={l} h={h}"
-                    assert (vb[b, h, :n + w.ws] == ref["vb"][l][b][h]).all(), f"V bytes differ l={l} h={h}"
+                    rk = ref["rank"][l][b][h]
+                    assert (kb[b, h, :n + w.ws] == U.buffer_order(ref["kb"][l][b][h], rk, n)).all(), f"K bytes differ l={l} h={h}"
+                    assert (vb[b, h, :n + w.ws] == U.buffer_order(ref["vb"][l][b][h], rk, n)).all(), f"V bytes differ l={l} h={h}"
     print(f"[{w.name}] max rel score error {worst:.2e}; near-tie events {near}; counts {g.counts.tolist()}")
     return near
 
@@ -187,7 +189,7 @@ def test_full_size_pass_sampled(name):
             got = g.scores(l)[b, h]
             U.assert_scores_close(got, ref, f"{name} l={l} b={b} h={h}")
             n = int(g.counts[b, l])
-            idx, _ = g.idx_rank(l)
+            idx, _ = g.kept(l)
             _, ev = U.select_matches(ref, idx[b, h, :n], n)
             near += ev
         print(f"[{name}] sampled heads ok; near-tie events {near}; counts {g.counts.tolist()}")
@@ -195,7 +197,7 @@ def test_full_size_pass_sampled(name):
             mask = synth.needle_token_mask(w)
             frac = []
             for l in range(w.L):
-                idx, _ = g.idx_rank(l)
+                idx, _ = g.kept(l)
                 n = int(g.counts[0, l])
                 frac.append(float(np.mean([mask[idx[0, h, :n]].sum() / 128.0 for h in range(w.Hkv)])))
             print("[needle32k] needle tokens retained per layer:", np.round(frac, 2).tolist())

@@ -232,7 +232,8 @@ def test_gather_and_shrink_bytes(D):
             got_k = kb[l].cpu().numpy().view(np.uint16)
             for b in range(w.Bt):
                 for h in range(w.Hkv):
-                    ref = O.gather_rows(kfull[l][b, h], O.select_topk(hist[l][b, h].astype(np.float64), w.Bl)["idx"], w.ws)
+                    first = O.select_topk(hist[l][b, h].astype(np.float64), w.Bl)
+                    ref = U.buffer_order(O.gather_rows(kfull[l][b, h], first["idx"], w.ws), first["rank"], w.Blc)
                     assert (got_k[b, h] == ref).all()
         counts = torch.empty((w.Bt, w.L), dtype=torch.int32, device="cuda")
         B.dkv_rebudget(c.h, w.L, counts)
@@ -247,10 +248,10 @@ def test_gather_and_shrink_bytes(D):
             got_v = vb[l].cpu().numpy().view(np.uint16)
             _, idx_a = B.dkv_layer_views(c.h, l)
             idx_now = B.read_device_i32(c.h, idx_a, (w.Bt, w.Hkv, w.Blc))
-            rank_dev = torch.zeros((w.Bt, w.Hkv, w.Blc), dtype=torch.int32, device="cuda")
-            B.dkv_ranks(c.h, l, rank_dev)
+            sorted_dev = torch.zeros((w.Bt, w.Hkv, w.Blc), dtype=torch.int32, device="cuda")
+            B.dkv_kept_sorted(c.h, l, sorted_dev)
             torch.cuda.synchronize()
-            rank_now = rank_dev.cpu().numpy()
+            sorted_now = sorted_dev.cpu().numpy()
             for b in range(w.Bt):
                 n = int(counts[b, l])
                 for h in range(w.Hkv):
@@ -259,8 +260,10 @@ def test_gather_and_shrink_bytes(D):
                     rk, ri, rr = O.shrink_rows(buf0, first["idx"], first["rank"], w.Blc, n, w.ws)
                     rv, _, _ = O.shrink_rows(O.gather_rows(vfull[l][b, h], first["idx"], w.ws), first["idx"],
                                              first["rank"], w.Blc, n, w.ws)
-                    assert (got_k[b, h, :n + w.ws] == rk).all() and (got_v[b, h, :n + w.ws] == rv).all()
-                    assert (idx_now[b, h, :n] == ri).all() and (rank_now[b, h, :n] == rr).all()
+                    assert (got_k[b, h, :n + w.ws] == U.buffer_order(rk, rr, n)).all()
+                    assert (got_v[b, h, :n + w.ws] == U.buffer_order(rv, rr, n)).all()
+                    assert (idx_now[b, h, :n] == ri[np.argsort(rr, kind="stable")]).all()
+                    assert (sorted_now[b, h, :n] == ri).all()
         # a second shrink with unchanged counts must leave everything as it is
         before = [t.clone() for t in kb]
         B.dkv_compact_all(c.h, w.L, kb, vb)
@@ -288,5 +291,6 @@ def test_gather_after_an_update_applies_the_new_count():
             torch.cuda.synchronize()
             n = int(counts[0, l])
             for h in range(2):
-                ref = O.gather_rows(kfull[l][0, h], O.select_topk(hist[l][0, h].astype(np.float64), n)["idx"], w.ws)
+                sel_n = O.select_topk(hist[l][0, h].astype(np.float64), n)
+                ref = U.buffer_order(O.gather_rows(kfull[l][0, h], sel_n["idx"], w.ws), sel_n["rank"], n)
                 assert (kb.cpu().numpy().view(np.uint16)[0, h, :n + w.ws] == ref).all()
