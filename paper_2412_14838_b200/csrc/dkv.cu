@@ -44,8 +44,8 @@ struct dkv_ctx {
   // tensor-core scoring
   int n_sms, tc_grid, tc_slots;
   float2* d_tc_stats;   // [3][Bt*Hkv][tc_slots][256]: partial softmax statistics, three layers in rotation
-  cudaStream_t side;    // second stream of dkv_run_prefill_pass (select / gather / rebudget / shrink)
-  cudaEvent_t ev_fork, ev_join, ev_scored[DKV_MAX_LAYERS];
+  cudaStream_t side[2]; // side streams of dkv_run_prefill_pass (select / gather / rebudget / shrink), layers alternate
+  cudaEvent_t ev_fork, ev_join[2], ev_update, ev_scored[DKV_MAX_LAYERS], ev_selected[DKV_MAX_LAYERS];
   // host state
   uint8_t scored[DKV_MAX_LAYERS], selected[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
   long long launches;
@@ -319,16 +319,16 @@ int do_reset(dkv_ctx* c, cudaStream_t st) {
 
 // Algorithm 1's loop.  The scoring launches run back to back on `st` (launch l = sweep 1 of layer l
 // followed by sweep 2 of layer l-1); everything that consumes a layer's scores (select, gather, and
-// every m layers rebudget + shrink) runs on the context's second stream behind an event, so that it
-// overlaps the scoring of the following layers.  `st` rejoins the second stream at the end.
+// every m layers rebudget + shrink) runs on two side streams, layers alternating between them, behind
+// events, so that it overlaps the scoring of the following layers.  `st` rejoins both at the end.
 int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* const* v, void* const* kb,
             void* const* vb, cudaStream_t st) {
   const Shape& s = c->s;
   int rc = do_reset(c, st);
   if (rc) return rc;
-  cudaStream_t sd = c->side;
   DKV_CUDA(c, cudaEventRecord(c->ev_fork, st));
-  DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_fork, 0));
+  for (int i = 0; i < 2; ++i) DKV_CUDA(c, cudaStreamWaitEvent(c->side[i], c->ev_fork, 0));
+  bool updated = false;
   for (int l = 0; l <= s.L; ++l) {
     const int sl = l < s.L ? l : -1, el = l - 1;
     if ((rc = launch_score(c, sl, sl >= 0 ? q[sl] : nullptr, sl >= 0 ? k[sl] : nullptr, el, el >= 0 ? q[el] : nullptr,
@@ -336,18 +336,27 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
       return rc;
     if (el < 0) continue;
     c->scored[el] = 1;
+    cudaStream_t sd = c->side[el & 1];
     DKV_CUDA(c, cudaEventRecord(c->ev_scored[el], st));
     DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_scored[el], 0));
     if ((rc = do_select(c, el, nullptr, nullptr, sd))) return rc;
     if ((rc = do_gather(c, el, k[el], v[el], kb[el], vb[el], sd))) return rc;
+    DKV_CUDA(c, cudaEventRecord(c->ev_selected[el], sd));
     const bool update = ((el + 1) % s.m == 0) || (el + 1 == s.L && s.L % s.m != 0);
     if (update) {
+      // needs every earlier layer selected and gathered (the other side stream) and the previous update
+      if (el >= 1) DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_selected[el - 1], 0));
+      if (updated) DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_update, 0));
       if ((rc = do_rebudget(c, el + 1, nullptr, sd))) return rc;
       if ((rc = do_shrink(c, 0, el + 1, kb, vb, sd))) return rc;
+      DKV_CUDA(c, cudaEventRecord(c->ev_update, sd));
+      updated = true;
     }
   }
-  DKV_CUDA(c, cudaEventRecord(c->ev_join, sd));
-  DKV_CUDA(c, cudaStreamWaitEvent(st, c->ev_join, 0));
+  for (int i = 0; i < 2; ++i) {
+    DKV_CUDA(c, cudaEventRecord(c->ev_join[i], c->side[i]));
+    DKV_CUDA(c, cudaStreamWaitEvent(st, c->ev_join[i], 0));
+  }
   return DKV_OK;
 }
 
@@ -356,10 +365,16 @@ void free_all(dkv_ctx* c) {
   cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_rb_state); cudaFree(c->d_rb_above); cudaFree(c->d_rb_hist1);
   cudaFree(c->d_rb_above2); cudaFree(c->d_rb_hist2); cudaFree(c->d_head_hist); cudaFree(c->d_head_offs);
   cudaFree(c->d_grouped); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
-  if (c->side) cudaStreamDestroy(c->side);
+  for (int i = 0; i < 2; ++i) {
+    if (c->side[i]) cudaStreamDestroy(c->side[i]);
+    if (c->ev_join[i]) cudaEventDestroy(c->ev_join[i]);
+  }
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
-  if (c->ev_join) cudaEventDestroy(c->ev_join);
-  for (int l = 0; l < DKV_MAX_LAYERS; ++l) if (c->ev_scored[l]) cudaEventDestroy(c->ev_scored[l]);
+  if (c->ev_update) cudaEventDestroy(c->ev_update);
+  for (int l = 0; l < DKV_MAX_LAYERS; ++l) {
+    if (c->ev_scored[l]) cudaEventDestroy(c->ev_scored[l]);
+    if (c->ev_selected[l]) cudaEventDestroy(c->ev_selected[l]);
+  }
   if (c->prof_recs) {
     for (ProfRec& r : *c->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     delete c->prof_recs;
@@ -442,7 +457,7 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
     const int tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
     const long long total_tiles = (long long)heads * tph;
     // leave a few SMs to the per-head select CTAs that dkv_run_prefill_pass runs beside the scoring
-    int side = heads < c->n_sms / 8 ? heads : c->n_sms / 8;
+    int side = 2 * heads < c->n_sms / 6 ? 2 * heads : c->n_sms / 6;
     if (const char* e = getenv("DKV_SIDE_SMS")) side = atoi(e);
     int score_sms = c->n_sms - side;
     if (score_sms < 1) score_sms = 1;
@@ -472,10 +487,16 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMalloc(&c->d_grouped, sizeof(uint32_t) * s.L * layer_scores(s)));
   TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * 3 * heads * c->tc_slots * 256));
   TRY(cudaFuncSetAttribute(tc::score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
-  TRY(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
+  for (int i = 0; i < 2; ++i) {
+    TRY(cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking));
+    TRY(cudaEventCreateWithFlags(&c->ev_join[i], cudaEventDisableTiming));
+  }
   TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
-  TRY(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
-  for (int l = 0; l < s.L; ++l) TRY(cudaEventCreateWithFlags(&c->ev_scored[l], cudaEventDisableTiming));
+  TRY(cudaEventCreateWithFlags(&c->ev_update, cudaEventDisableTiming));
+  for (int l = 0; l < s.L; ++l) {
+    TRY(cudaEventCreateWithFlags(&c->ev_scored[l], cudaEventDisableTiming));
+    TRY(cudaEventCreateWithFlags(&c->ev_selected[l], cudaEventDisableTiming));
+  }
   TRY(cudaMalloc(&c->d_status, sizeof(int) * 8));
   TRY(cudaMemset(c->d_status, 0, sizeof(int) * 8));
   TRY(cudaMemset(c->d_count, 0, sizeof(int) * bl));

@@ -86,12 +86,17 @@ __device__ __forceinline__ unsigned int agg_bump(unsigned int* counters, unsigne
   return base + (unsigned int)__popc(peers & ((1u << lane) - 1u));
 }
 
-// Bitonic sort of keys[0 .. sort_n) ascending; sort_n a power of two.  Ends with a barrier.
+// Bitonic sort of keys[0 .. sort_n) ascending; sort_n a power of two >= 2.  Strides of 64 and more are
+// done by the whole block with a barrier per stage; the strides below that stay inside 64-key blocks,
+// each owned by one warp, and only need warp barriers.  Ends with a block barrier.
 __device__ __forceinline__ void bitonic_sort(unsigned long long* keys, int sort_n) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int blk = sort_n < 64 ? sort_n : 64;               // keys per warp-owned block
   for (int size = 2; size <= sort_n; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+    int stride = size >> 1;
+    for (; stride >= 64; stride >>= 1) {
       for (int t = threadIdx.x; t < (sort_n >> 1); t += blockDim.x) {
-        const int lo = ((t / stride) * stride * 2) + (t % stride);
+        const int lo = ((t & ~(stride - 1)) << 1) | (t & (stride - 1));
         const int hi = lo + stride;
         const bool up = ((lo & size) == 0);
         const unsigned long long a = keys[lo], b = keys[hi];
@@ -99,6 +104,19 @@ __device__ __forceinline__ void bitonic_sort(unsigned long long* keys, int sort_
       }
       __syncthreads();
     }
+    for (int base = warp * blk; base < sort_n; base += nwarps * blk) {
+      for (int s = stride; s > 0; s >>= 1) {
+        if (lane < (blk >> 1)) {
+          const int lo = base + (((lane & ~(s - 1)) << 1) | (lane & (s - 1)));
+          const int hi = lo + s;
+          const bool up = ((lo & size) == 0);
+          const unsigned long long a = keys[lo], b = keys[hi];
+          if ((a > b) == up) { keys[lo] = b; keys[hi] = a; }
+        }
+        __syncwarp();
+      }
+    }
+    __syncthreads();
   }
 }
 
@@ -124,7 +142,8 @@ select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int*
   const uint32_t* v = reinterpret_cast<const uint32_t*>(scores) + (size_t)blockIdx.x * P;
   if (tid == 0 && blockIdx.x % Hkv == 0) count[(blockIdx.x / Hkv) * L + layer] = keep;
 
-  const size_t stage_bytes = ((REG ? (size_t)P * 4 : 0) > (size_t)sort_n * 8 ? (size_t)P * 4 : (size_t)sort_n * 8);
+  size_t stage_bytes = (size_t)sort_n * 8;
+  if (REG && (size_t)P * 4 > stage_bytes) stage_bytes = (size_t)P * 4;
   uint32_t* stage = reinterpret_cast<uint32_t*>(dyn);                       // grouped scores (REG), later sort keys
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(dyn);
   int* sel_pos = reinterpret_cast<int*>(dyn + ((stage_bytes + 15) & ~(size_t)15));
@@ -139,7 +158,9 @@ select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int*
   }
 #define DKV_SEL_FOR(e) _Pragma("unroll") for (int e = 0; e < n_e; ++e)
 #define DKV_SEL_POS(e) (run0 + (e) * 32 + lane)
-#define DKV_SEL_OK(e) ((e) < chunk && DKV_SEL_POS(e) < P)
+  // which of this lane's slots hold a position: slots [0, n_ok)
+  const int n_ok = min(chunk, max(0, (P - run0 - lane + 31) / 32));
+#define DKV_SEL_OK(e) ((e) < n_ok)
   auto val = [&](int e) -> uint32_t {
     if constexpr (REG) return r[e]; else return DKV_SEL_OK(e) ? v[DKV_SEL_POS(e)] : 0u;
   };
