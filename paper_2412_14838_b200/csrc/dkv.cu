@@ -189,17 +189,18 @@ bool make_job(dkv_ctx* c, int mode, int layer, const void* q, const void* k, flo
   return true;
 }
 
-// One launch: sweep 1 of `stats_layer` (if >= 0), then sweep 2 of `emit_layer` (if >= 0).
+// One launch: sweep 2 of `emit_layer` (if >= 0), then sweep 1 of `stats_layer` (if >= 0).  In the pass the
+// emit layer is the one whose keys the previous launch streamed last, so its second read finds them in L2.
 int launch_score(dkv_ctx* c, int stats_layer, const void* sq, const void* sk, int emit_layer, const void* eq,
                  const void* ek, float* scores_out, cudaStream_t st) {
   CUtensorMap qm0, km0, qm1, km1;
   tc::Params j0, j1;
   memset(&j0, 0, sizeof j0); memset(&j1, 0, sizeof j1);
   j0.mode = j1.mode = tc::kNone;
-  if (stats_layer >= 0 && !make_job(c, tc::kStats, stats_layer, sq, sk, nullptr, stats_layer % 3, &qm0, &km0, &j0)) return DKV_ERR_CUDA;
-  if (emit_layer >= 0 && !make_job(c, tc::kEmit, emit_layer, eq, ek, scores_out, emit_layer % 3, &qm1, &km1, &j1)) return DKV_ERR_CUDA;
-  if (stats_layer < 0) { qm0 = qm1; km0 = km1; }
-  if (emit_layer < 0) { qm1 = qm0; km1 = km0; }
+  if (emit_layer >= 0 && !make_job(c, tc::kEmit, emit_layer, eq, ek, scores_out, emit_layer % 3, &qm0, &km0, &j0)) return DKV_ERR_CUDA;
+  if (stats_layer >= 0 && !make_job(c, tc::kStats, stats_layer, sq, sk, nullptr, stats_layer % 3, &qm1, &km1, &j1)) return DKV_ERR_CUDA;
+  if (emit_layer < 0) { qm0 = qm1; km0 = km1; }
+  if (stats_layer < 0) { qm1 = qm0; km1 = km0; }
   ProfScope ps(c, stats_layer >= 0 ? DKV_STEP_SCORE_STATS : DKV_STEP_SCORE_EMIT, 1, st);
   tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm0, km0, qm1, km1, j0, j1);
   DKV_LAUNCHED(c);
