@@ -2,11 +2,12 @@
 // so far, the number of top-K hits per layer, then the integer budget arithmetic.
 //
 // Only per-layer counts leave the selection.  Every head's scores were histogrammed by their first
-// 11-bit digit and stored grouped by that digit when the layer was selected (select.cuh), so:
+// 11-bit digit when the layer was selected (select.cuh), so:
 //   rb_locate   adds up the per-head histograms of layers [0, l), finds the digit b* that holds the K-th
 //               largest score, and reads each layer's count of scores above b* off the offsets;
-//   rb_refine1  histograms the next 11 bits of the scores inside bucket b* (the only scores read);
-//   rb_refine2  counts, per layer, the bucket's scores above the second digit and histograms the last
+//   rb_refine1  streams the history once, copies the scores whose first digit is b* (with their layer)
+//               into a candidate list and histograms their next 11 bits;
+//   rb_refine2  counts, per layer, the candidates above the second digit and histograms the last
 //               10 bits of those that match it;
 //   rb_budget   fixes the exact threshold T, gives the entries equal to T to the lowest layers first
 //               (flat-index tie rule), and evaluates Eq. 5-6 in exact integers.
@@ -27,11 +28,11 @@ struct RbState {          // per sample
 
 // One CTA of 1024 threads per sample.
 // head_hist/head_offs: [L][Bt][Hkv][2048].  above: [Bt][L] scores above bucket b* per layer.
-// hist1: [Bt][2048], above2: [Bt][L], hist2: [Bt][L][1024] are cleared here for the refine kernels.
+// hist1: [Bt][2048], above2: [Bt][L], hist2: [Bt][L][1024], cand_n: [Bt] are cleared here for the refine kernels.
 __global__ void __launch_bounds__(1024)
 rb_locate_kernel(const unsigned int* __restrict__ head_hist, const unsigned int* __restrict__ head_offs,
                  RbState* __restrict__ state, unsigned int* __restrict__ above, unsigned int* __restrict__ hist1,
-                 unsigned int* __restrict__ above2, unsigned int* __restrict__ hist2,
+                 unsigned int* __restrict__ above2, unsigned int* __restrict__ hist2, unsigned int* __restrict__ cand_n,
                  int Bt, int Hkv, int L, int l, int P, long long k) {
   __shared__ unsigned int hist[kBins];
   __shared__ int sm_scan[33];
@@ -54,6 +55,7 @@ rb_locate_kernel(const unsigned int* __restrict__ head_hist, const unsigned int*
     atomicAdd(hb + 0, a0.x); atomicAdd(hb + 1, a0.y); atomicAdd(hb + 2, a0.z); atomicAdd(hb + 3, a0.w);
     atomicAdd(hb + 4, a1.x); atomicAdd(hb + 5, a1.y); atomicAdd(hb + 6, a1.z); atomicAdd(hb + 7, a1.w);
   }
+  if (tid == 0) cand_n[b] = 0;
   for (int e = tid; e < L; e += 1024) above2[b * L + e] = 0;
   for (int e = tid; e < l * 1024; e += 1024) hist2[(size_t)b * L * 1024 + e] = 0;
   __syncthreads();
@@ -71,59 +73,70 @@ rb_locate_kernel(const unsigned int* __restrict__ head_hist, const unsigned int*
   }
 }
 
-// grid (slices, l * Hkv, Bt): second-digit histogram of the scores in bucket b*.
+// grid (slices, l, Bt): one pass over the scores of layers [0, l).  Scores whose first digit is b* go to the
+// sample's candidate list (value, layer) and into the second-digit histogram.  The list has room for every
+// score (cand[b] holds l*Hkv*P pairs at most); its order is arbitrary, only counts are taken from it.
 __global__ void __launch_bounds__(kRbThreads)
-rb_refine1_kernel(const uint32_t* __restrict__ grouped, const unsigned int* __restrict__ head_hist,
-                  const unsigned int* __restrict__ head_offs, const RbState* __restrict__ state,
-                  unsigned int* __restrict__ hist1, int Bt, int Hkv, int P) {
+rb_refine1_kernel(const float* __restrict__ scores, const RbState* __restrict__ state, unsigned int* __restrict__ hist1,
+                  uint2* __restrict__ cand, unsigned int* __restrict__ cand_n, int Bt, size_t per_layer /* Hkv*P */,
+                  size_t cand_stride) {
   __shared__ unsigned int sh[kBins];
-  const int b = blockIdx.z, i = blockIdx.y / Hkv, h = blockIdx.y % Hkv;
-  const int d = state[b].bstar;
-  const size_t head = ((size_t)i * Bt + b) * Hkv + h;
-  const int n = (int)head_hist[head * kBins + d];
-  if ((int)(blockIdx.x * kRbThreads) >= n) return;
-  const uint32_t* src = grouped + head * P + head_offs[head * kBins + d];
+  __shared__ unsigned int s_cnt, s_base;
+  const int b = blockIdx.z, i = blockIdx.y;
+  const uint32_t d = (uint32_t)state[b].bstar;
+  const uint32_t* v = reinterpret_cast<const uint32_t*>(scores) + ((size_t)i * Bt + b) * per_layer;
   for (int j = threadIdx.x; j < kBins; j += kRbThreads) sh[j] = 0;
+  if (threadIdx.x == 0) s_cnt = 0;
   __syncthreads();
-  for (int e = blockIdx.x * kRbThreads + threadIdx.x; e < n; e += gridDim.x * kRbThreads)
-    atomicAdd(&sh[(src[e] >> 10) & 2047u], 1u);
+  // two sweeps over this block's slice: count, reserve a range of the list, then fill it
+  const size_t per_block = (per_layer + gridDim.x - 1) / gridDim.x;
+  const size_t e0 = (size_t)blockIdx.x * per_block, e1 = e0 + per_block < per_layer ? e0 + per_block : per_layer;
+  unsigned int mine = 0;
+  for (size_t e = e0 + threadIdx.x; e < e1; e += kRbThreads) mine += ((v[e] >> 21) == d);
+  if (mine) atomicAdd(&s_cnt, mine);
+  __syncthreads();
+  const unsigned int block_total = s_cnt;
+  __syncthreads();
+  if (block_total == 0) return;
+  if (threadIdx.x == 0) { s_base = atomicAdd(&cand_n[b], block_total); s_cnt = 0; }
+  __syncthreads();
+  uint2* list = cand + (size_t)b * cand_stride;
+  for (size_t e = e0 + threadIdx.x; e < e1; e += kRbThreads) {
+    const uint32_t u = v[e];
+    if ((u >> 21) == d) {
+      list[s_base + atomicAdd(&s_cnt, 1u)] = make_uint2(u, (unsigned int)i);
+      atomicAdd(&sh[(u >> 10) & 2047u], 1u);
+    }
+  }
   __syncthreads();
   for (int j = threadIdx.x; j < kBins; j += kRbThreads) { const unsigned int c = sh[j]; if (c) atomicAdd(&hist1[(size_t)b * kBins + j], c); }
 }
 
-// Same grid.  Every block re-derives the second digit s* from hist1; then per layer: bucket scores with a
-// larger second digit (above2) and the last-10-bit histogram of those with second digit s* (hist2).
+// grid (slices, Bt) over the candidate list.  Every block re-derives the second digit s* from hist1; then per
+// layer: candidates with a larger second digit (above2) and the last-10-bit histogram of those with second
+// digit s* (hist2).
 __global__ void __launch_bounds__(kRbThreads)
-rb_refine2_kernel(const uint32_t* __restrict__ grouped, const unsigned int* __restrict__ head_hist,
-                  const unsigned int* __restrict__ head_offs, const RbState* __restrict__ state,
+rb_refine2_kernel(const uint2* __restrict__ cand, const unsigned int* __restrict__ cand_n, const RbState* __restrict__ state,
                   const unsigned int* __restrict__ hist1, unsigned int* __restrict__ above2,
-                  unsigned int* __restrict__ hist2, int Bt, int Hkv, int L, int P) {
+                  unsigned int* __restrict__ hist2, int L, size_t cand_stride) {
   __shared__ unsigned int sh[kBins];
   __shared__ int sm_scan[33];
   __shared__ int found[2];
-  __shared__ unsigned int s_above;
-  const int b = blockIdx.z, i = blockIdx.y / Hkv, h = blockIdx.y % Hkv;
+  const int b = blockIdx.y;
   const RbState st = state[b];
-  const size_t head = ((size_t)i * Bt + b) * Hkv + h;
-  const int n = (int)head_hist[head * kBins + st.bstar];
-  if ((int)(blockIdx.x * kRbThreads) >= n) return;
+  const unsigned int n = cand_n[b];
+  if (blockIdx.x * kRbThreads >= n) return;
   for (int j = threadIdx.x; j < kBins; j += kRbThreads) sh[j] = hist1[(size_t)b * kBins + j];
-  if (threadIdx.x == 0) s_above = 0;
   __syncthreads();
   find_digit(sh, kBins, st.cand, st.need1, sm_scan, found, nullptr);
   const uint32_t s2 = (uint32_t)found[0];
-  const uint32_t* src = grouped + head * P + head_offs[head * kBins + st.bstar];
-  unsigned int mine = 0;
-  for (int e = blockIdx.x * kRbThreads + threadIdx.x; e < n; e += gridDim.x * kRbThreads) {
-    const uint32_t u = src[e], dd = (u >> 10) & 2047u;
-    if (dd > s2) ++mine;
-    else if (dd == s2) atomicAdd(&hist2[((size_t)b * L + i) * 1024 + (u & 1023u)], 1u);
+  const uint2* list = cand + (size_t)b * cand_stride;
+  for (unsigned int e = blockIdx.x * kRbThreads + threadIdx.x; e < n; e += gridDim.x * kRbThreads) {
+    const uint2 c = list[e];
+    const uint32_t dd = (c.x >> 10) & 2047u;
+    if (dd > s2) atomicAdd(&above2[b * L + c.y], 1u);
+    else if (dd == s2) atomicAdd(&hist2[((size_t)b * L + c.y) * 1024 + (c.x & 1023u)], 1u);
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
-  if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&s_above, mine);
-  __syncthreads();
-  if (threadIdx.x == 0 && s_above) atomicAdd(&above2[b * L + i], s_above);
 }
 
 // One CTA of 1024 threads per sample: exact T, per-layer hits, Eq. 5-6.

@@ -9,9 +9,8 @@
 // position ascending): that is the order Algorithm 1's topk() returns and stores them in, and a
 // later truncation to a smaller budget is a prefix of it.
 // The first pass's histogram (top 11 bits: sign, exponent, 2 mantissa bits) is also kept per head
-// in global memory, together with a copy of the head's scores grouped by that digit, so that
-// Update_Buffer_Length can locate the global K-th value from histograms and then look only at
-// the one bucket that contains it, instead of re-reading every layer's scores at every update.
+// in global memory with its prefix offsets, so that Update_Buffer_Length can locate the first digit
+// of the global K-th value, and each layer's count of scores above it, from histograms alone.
 #pragma once
 #include "common.cuh"
 
@@ -124,16 +123,14 @@ __device__ __forceinline__ void bitonic_sort(unsigned long long* keys, int sort_
 // idx: [Bt*Hkv][keep] kept positions in buffer order = (score descending, position ascending).
 // sorted_out (optional): the same positions ascending; rank_out (optional): rank of each of those.
 // head_hist, head_offs: [Bt*Hkv][2048] first-digit counts of the head and their ascending exclusive offsets.
-// grouped: [Bt*Hkv][P] the head's score bits grouped by first digit (ascending digit; order inside a
-// group is unspecified).  Also records count[b][layer] = keep.
+// Also records count[b][layer] = keep.
 // Every warp owns a run of 32*chunk consecutive positions; lane j holds positions run + 32*e + j.
-// Dynamic shared memory: max(REG ? 4*P : 0, 8*sort_n) bytes rounded up to 16, then 4*keep bytes.
+// Dynamic shared memory: 8*sort_n bytes, then 4*keep bytes.
 template <bool REG>
 __global__ void __launch_bounds__(kSelThreads)
 select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int* __restrict__ sorted_out,
                    int* __restrict__ rank_out, unsigned int* __restrict__ head_hist, unsigned int* __restrict__ head_offs,
-                   uint32_t* __restrict__ grouped, int P, int keep, int sort_n, int* __restrict__ count, int Hkv, int L,
-                   int layer) {
+                   int P, int keep, int sort_n, int* __restrict__ count, int Hkv, int L, int layer) {
   extern __shared__ __align__(16) unsigned char dyn[];
   __shared__ unsigned int hist[kBins];
   __shared__ int sm_scan[33], sm_scan2[33];
@@ -142,69 +139,53 @@ select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int*
   const uint32_t* v = reinterpret_cast<const uint32_t*>(scores) + (size_t)blockIdx.x * P;
   if (tid == 0 && blockIdx.x % Hkv == 0) count[(blockIdx.x / Hkv) * L + layer] = keep;
 
-  size_t stage_bytes = (size_t)sort_n * 8;
-  if (REG && (size_t)P * 4 > stage_bytes) stage_bytes = (size_t)P * 4;
-  uint32_t* stage = reinterpret_cast<uint32_t*>(dyn);                       // grouped scores (REG), later sort keys
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(dyn);
-  int* sel_pos = reinterpret_cast<int*>(dyn + ((stage_bytes + 15) & ~(size_t)15));
+  int* sel_pos = reinterpret_cast<int*>(dyn + (size_t)sort_n * 8);
 
   const int chunk = (P + kSelThreads - 1) / kSelThreads;       // REG: chunk <= kRegChunk
   const int run0 = warp * chunk * 32;
   const int n_e = REG ? kRegChunk : chunk;
+  // which of this lane's slots hold a position: slots [0, n_ok)
+  const int n_ok = min(chunk, max(0, (P - run0 - lane + 31) / 32));
   uint32_t r[REG ? kRegChunk : 1];
   if constexpr (REG) {
 #pragma unroll
-    for (int e = 0; e < kRegChunk; ++e) { const int p = run0 + e * 32 + lane; r[e] = (e < chunk && p < P) ? v[p] : 0u; }
+    for (int e = 0; e < kRegChunk; ++e) r[e] = e < n_ok ? v[run0 + e * 32 + lane] : 0u;
   }
 #define DKV_SEL_FOR(e) _Pragma("unroll") for (int e = 0; e < n_e; ++e)
 #define DKV_SEL_POS(e) (run0 + (e) * 32 + lane)
-  // which of this lane's slots hold a position: slots [0, n_ok)
-  const int n_ok = min(chunk, max(0, (P - run0 - lane + 31) / 32));
 #define DKV_SEL_OK(e) ((e) < n_ok)
   auto val = [&](int e) -> uint32_t {
     if constexpr (REG) return r[e]; else return DKV_SEL_OK(e) ? v[DKV_SEL_POS(e)] : 0u;
   };
 
-  uint32_t prefix = 0, mask = 0;
-  int need = keep, total = P;
-  for (int pass = 0; pass < 3; ++pass) {
+  // pass 0: first digit of every score; neighbours share digits after pooling, so lanes combine their bumps
+  for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
+  __syncthreads();
+  DKV_SEL_FOR(e) agg_bump(hist, val(e) >> 21, DKV_SEL_OK(e));
+  __syncthreads();
+  {
+    unsigned int* gh = head_hist + (size_t)blockIdx.x * kBins;
+    for (int i = tid; i < kBins; i += kSelThreads) gh[i] = hist[i];
+  }
+  find_digit(hist, kBins, P, keep, sm_scan, found, head_offs + (size_t)blockIdx.x * kBins);
+  uint32_t prefix = ((uint32_t)found[0]) << 21, mask = 2047u << 21;
+  int need = found[1], total = (int)hist[found[0]];
+  __syncthreads();
+  // passes 1, 2: only the scores inside the first digit's bucket take part
+  for (int pass = 1; pass < 3; ++pass) {
     const int shift = digit_shift(pass);
     const uint32_t dm = digit_mask(pass);
     for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
     __syncthreads();
     DKV_SEL_FOR(e) {
       const uint32_t u = val(e);
-      const bool in = DKV_SEL_OK(e) && (u & mask) == prefix;
-      if (pass == 0) agg_bump(hist, (u >> shift) & dm, in);          // neighbours share digits after pooling
-      else if (in) atomicAdd(&hist[(u >> shift) & dm], 1u);
+      if (DKV_SEL_OK(e) && (u & mask) == prefix) atomicAdd(&hist[(u >> shift) & dm], 1u);
     }
     __syncthreads();
-    if (pass == 0) {
-      unsigned int* gh = head_hist + (size_t)blockIdx.x * kBins;
-      for (int i = tid; i < kBins; i += kSelThreads) gh[i] = hist[i];
-    }
-    find_digit(hist, kBins, total, need, sm_scan, found, pass == 0 ? head_offs + (size_t)blockIdx.x * kBins : nullptr);
+    find_digit(hist, kBins, total, need, sm_scan, found, nullptr);
     const int d = found[0];
-    const int cnt_d = (int)hist[d];
-    if (pass == 0) {
-      // group the head's scores by first digit: cursor[d] starts at the digit's offset
-      const unsigned int* go = head_offs + (size_t)blockIdx.x * kBins;
-      __syncthreads();
-      for (int i = tid; i < kBins; i += kSelThreads) hist[i] = go[i];
-      __syncthreads();
-      uint32_t* dst = grouped + (size_t)blockIdx.x * P;
-      DKV_SEL_FOR(e) {
-        const uint32_t u = val(e);
-        const bool in = DKV_SEL_OK(e);
-        const unsigned int slot = agg_bump(hist, u >> 21, in);
-        if (in) { if constexpr (REG) stage[slot] = u; else dst[slot] = u; }
-      }
-      if constexpr (REG) {
-        __syncthreads();
-        for (int i = tid; i < P; i += kSelThreads) dst[i] = stage[i];
-      }
-    }
-    total = cnt_d;
+    total = (int)hist[d];
     need = found[1];
     prefix |= ((uint32_t)d) << shift;
     mask |= dm << shift;
@@ -230,15 +211,17 @@ select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int*
     const bool ok = DKV_SEL_OK(e);
     const bool is_gt = ok && u > T, is_eq = ok && u == T;
     const unsigned int bg = __ballot_sync(0xFFFFFFFFu, is_gt), be = __ballot_sync(0xFFFFFFFFu, is_eq);
-    const int g = g_run + __popc(bg & lt), q = q_run + __popc(be & lt);
-    if (is_gt || (is_eq && q < need_eq)) {
-      const int out = g + min(q, need_eq);
-      const int p = DKV_SEL_POS(e);
-      sel_pos[out] = p;
-      if (my_sorted) my_sorted[out] = p;
-      keys[out] = ((unsigned long long)(~u) << 32) | (unsigned int)out;
+    if (bg | be) {                           // warp-uniform: most rows of 32 positions keep nothing
+      const int g = g_run + __popc(bg & lt), q = q_run + __popc(be & lt);
+      if (is_gt || (is_eq && q < need_eq)) {
+        const int out = g + min(q, need_eq);
+        const int p = DKV_SEL_POS(e);
+        sel_pos[out] = p;
+        if (my_sorted) my_sorted[out] = p;
+        keys[out] = ((unsigned long long)(~u) << 32) | (unsigned int)out;
+      }
+      g_run += __popc(bg); q_run += __popc(be);
     }
-    g_run += __popc(bg); q_run += __popc(be);
   }
   for (int i = tid + keep; i < sort_n; i += kSelThreads) keys[i] = ~0ull;
   __syncthreads();
