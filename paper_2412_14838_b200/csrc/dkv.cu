@@ -13,7 +13,6 @@
 #include "compact.cuh"
 #include "rebudget.cuh"
 #include "score_tc.cuh"
-#include "score_fused.cuh"
 #include "select.cuh"
 
 using namespace dkv;
@@ -46,14 +45,6 @@ struct dkv_ctx {
   // tensor-core scoring
   int n_sms, tc_grid, tc_slots;
   float2* d_tc_stats;   // [3][Bt*Hkv][tc_slots][256]: partial softmax statistics, three layers in rotation
-  // single-sweep scoring (score_fused.cuh), used when the shape allows
-  bool fused_ok;
-  int f_pp, f_hpr, f_rounds;
-  unsigned int f_epoch;
-  float2* d_f_part;           // [Bt*Hkv][pp][128]
-  float* d_f_lse;             // [Bt*Hkv][128]
-  unsigned int* d_f_flags;    // done[heads], ready[heads], halo_flag[heads][pp]
-  float* d_f_halo;            // [Bt*Hkv][pp][2*kHaloMax]
   cudaStream_t side[2]; // side streams of dkv_run_prefill_pass (select / gather / rebudget / shrink), layers alternate
   cudaEvent_t ev_fork, ev_join[2], ev_update, ev_scored[DKV_MAX_LAYERS], ev_selected[DKV_MAX_LAYERS];
   // host state
@@ -217,41 +208,10 @@ int launch_score(dkv_ctx* c, int stats_layer, const void* sq, const void* sk, in
   return DKV_OK;
 }
 
-// Both sweeps of one layer in one launch, keys read once (score_fused.cuh).
-int launch_fused(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
-  const Shape& s = c->s;
-  const int heads = s.Bt * s.Hkv;
-  CUtensorMap qm, km;
-  if (!make_map(&qm, q, s.D, s.M, heads) || !make_map(&km, k, s.D, s.S, heads)) return DKV_ERR_CUDA;
-  tc::FusedParams p;
-  p.S = s.S; p.P = s.P; p.ws = s.ws; p.M = s.M; p.D = s.D; p.heads = heads; p.half = s.pool / 2;
-  p.tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
-  p.nq16 = (s.M + 15) / 16 * 16;
-  p.pp = c->f_pp; p.hpr = c->f_hpr; p.n_rounds = c->f_rounds;
-  p.scale2 = kLog2e / sqrtf((float)s.D);
-  p.idesc_stats = make_idesc(128, 128);
-  p.idesc_emit = make_idesc(128, p.nq16);
-  p.epoch = ++c->f_epoch;
-  p.part = c->d_f_part; p.lse = c->d_f_lse;
-  p.done = c->d_f_flags; p.ready = c->d_f_flags + heads; p.halo_flag = c->d_f_flags + 2 * heads;
-  p.halo_val = c->d_f_halo;
-  p.scores = c->d_scores + (size_t)layer * layer_scores(s);
-  p.copy_out = scores_out;
-  p.status = c->d_status;
-  ProfScope ps(c, DKV_STEP_SCORE_STATS, 1, st);
-  tc::score_fused_kernel<<<c->tc_grid, tc::kThreads, tc::kFusedSmemBytes, st>>>(qm, km, p);
-  DKV_LAUNCHED(c);
-  return DKV_OK;
-}
-
 int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
-  int rc;
-  if (c->fused_ok) {
-    if ((rc = launch_fused(c, layer, q, k, scores_out, st))) return rc;
-  } else {
-    if ((rc = launch_score(c, layer, q, k, -1, nullptr, nullptr, nullptr, st))) return rc;
-    if ((rc = launch_score(c, -1, nullptr, nullptr, layer, q, k, scores_out, st))) return rc;
-  }
+  int rc = launch_score(c, layer, q, k, -1, nullptr, nullptr, nullptr, st);
+  if (rc) return rc;
+  if ((rc = launch_score(c, -1, nullptr, nullptr, layer, q, k, scores_out, st))) return rc;
   c->scored[layer] = 1;
   c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
   return DKV_OK;
@@ -360,8 +320,8 @@ int do_reset(dkv_ctx* c, cudaStream_t st) {
   return DKV_OK;
 }
 
-// Algorithm 1's loop.  The scoring launches run back to back on `st` (one single-sweep launch per layer
-// where the shape allows it, else launch l = sweep 2 of layer l-1 followed by sweep 1 of layer l); everything that consumes a layer's scores (select, gather, and
+// Algorithm 1's loop.  The scoring launches run back to back on `st` (launch l = sweep 1 of layer l
+// followed by sweep 2 of layer l-1); everything that consumes a layer's scores (select, gather, and
 // every m layers rebudget + shrink) runs on two side streams, layers alternating between them, behind
 // events, so that it overlaps the scoring of the following layers.  `st` rejoins both at the end.
 int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* const* v, void* const* kb,
@@ -372,14 +332,11 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
   DKV_CUDA(c, cudaEventRecord(c->ev_fork, st));
   for (int i = 0; i < 2; ++i) DKV_CUDA(c, cudaStreamWaitEvent(c->side[i], c->ev_fork, 0));
   bool updated = false;
-  for (int l = c->fused_ok ? 1 : 0; l <= s.L; ++l) {
+  for (int l = 0; l <= s.L; ++l) {
     const int sl = l < s.L ? l : -1, el = l - 1;
-    if (c->fused_ok) {
-      if ((rc = launch_fused(c, el, q[el], k[el], nullptr, st))) return rc;
-    } else if ((rc = launch_score(c, sl, sl >= 0 ? q[sl] : nullptr, sl >= 0 ? k[sl] : nullptr, el,
-                                  el >= 0 ? q[el] : nullptr, el >= 0 ? k[el] : nullptr, nullptr, st))) {
+    if ((rc = launch_score(c, sl, sl >= 0 ? q[sl] : nullptr, sl >= 0 ? k[sl] : nullptr, el, el >= 0 ? q[el] : nullptr,
+                           el >= 0 ? k[el] : nullptr, nullptr, st)))
       return rc;
-    }
     if (el < 0) continue;
     c->scored[el] = 1;
     cudaStream_t sd = c->side[el & 1];
@@ -410,8 +367,7 @@ void free_all(dkv_ctx* c) {
   cudaFree(c->d_scores); cudaFree(c->d_idx); cudaFree(c->d_count);
   cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_rb_state); cudaFree(c->d_rb_above); cudaFree(c->d_rb_hist1);
   cudaFree(c->d_rb_above2); cudaFree(c->d_rb_hist2); cudaFree(c->d_head_hist); cudaFree(c->d_head_offs);
-  cudaFree(c->d_cand); cudaFree(c->d_cand_n); cudaFree(c->d_f_part); cudaFree(c->d_f_lse); cudaFree(c->d_f_flags);
-  cudaFree(c->d_f_halo); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
+  cudaFree(c->d_cand); cudaFree(c->d_cand_n); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
   for (int i = 0; i < 2; ++i) {
     if (c->side[i]) cudaStreamDestroy(c->side[i]);
     if (c->ev_join[i]) cudaEventDestroy(c->ev_join[i]);
@@ -516,12 +472,6 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
       if (hi - lo + 1 > slots) slots = hi - lo + 1;
     }
     c->tc_slots = slots;
-    // single-sweep scoring: window rows in one MMA block, a head's tile pairs within one round of the grid
-    c->f_pp = (tph + 1) / 2;
-    c->fused_ok = s.M <= 128 && c->f_pp <= c->tc_grid && s.pool / 2 < tc::kHaloMax && getenv("DKV_TWO_SWEEP") == nullptr;
-    c->f_hpr = c->fused_ok ? c->tc_grid / c->f_pp : 1;
-    c->f_rounds = (heads + c->f_hpr - 1) / c->f_hpr;
-    c->f_epoch = 0;
   }
   const size_t bl = (size_t)s.Bt * s.L;
 #define TRY(call) if (e == cudaSuccess) e = (call)
@@ -541,12 +491,6 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMalloc(&c->d_cand_n, sizeof(unsigned int) * s.Bt));
   TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * 3 * heads * c->tc_slots * 256));
   TRY(cudaFuncSetAttribute(tc::score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
-  TRY(cudaFuncSetAttribute(tc::score_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kFusedSmemBytes));
-  TRY(cudaMalloc(&c->d_f_part, sizeof(float2) * heads * c->f_pp * 128));
-  TRY(cudaMalloc(&c->d_f_lse, sizeof(float) * heads * 128));
-  TRY(cudaMalloc(&c->d_f_flags, sizeof(unsigned int) * heads * (2 + c->f_pp)));
-  TRY(cudaMemset(c->d_f_flags, 0, sizeof(unsigned int) * heads * (2 + c->f_pp)));
-  TRY(cudaMalloc(&c->d_f_halo, sizeof(float) * heads * c->f_pp * 2 * tc::kHaloMax));
   for (int i = 0; i < 2; ++i) {
     TRY(cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking));
     TRY(cudaEventCreateWithFlags(&c->ev_join[i], cudaEventDisableTiming));
