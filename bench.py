@@ -163,6 +163,23 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+# ------------------------------------------------------------------------------------ replicas
+def max_over_ranks(x: float, device: str = "cuda") -> float:
+    """The slowest rank's time: every rank runs an independent replica, the job ends with the last one."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_replica: int, world: int, seconds_per_step: float) -> float:
+    """Aggregate tokens/s of `world` independent replicas that all took `seconds_per_step` (the max)."""
+    return world * tokens_per_replica / seconds_per_step
+
+
 # ------------------------------------------------------------------------------------ GPU leg
 def run_gpu(args, w):
     import torch
@@ -221,13 +238,10 @@ def run_gpu(args, w):
         barrier()
     ms = ev0.elapsed_time(ev1)
     launches = B.dkv_launch_count(ctx) - launches0
-    tmax = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-    ms = float(tmax.item())
+    ms = max_over_ranks(ms)
     ms_per_step = ms / args.steps
     tokens = w.Bt * w.S
-    value = world * tokens / (ms_per_step * 1e-3)
+    value = whole_job_value(tokens, world, ms_per_step * 1e-3)
 
     # per-kernel durations: the same steps again, each step's launches bracketed by CUDA events
     B.dkv_profile(ctx, True)
@@ -266,13 +280,10 @@ def run_gpu(args, w):
             B.dkv_run_prefill_pass_host(ctx, hq, hk, hv, okb, ovb, counts)
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / e2e_steps
-        tdt = torch.tensor([dt], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(tdt, op=dist.ReduceOp.MAX)
-        dt = float(tdt.item())
+        dt = max_over_ranks(dt)
         h2d = sum(t.numel() * 2 for t in hq) + sum(t.numel() * 2 for t in hk) + sum(t.numel() * 2 for t in hv)
         d2h = sum(t.numel() * 2 for t in okb) + sum(t.numel() * 2 for t in ovb) + counts.nbytes
-        e2e = {"value": world * tokens / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+        e2e = {"value": whole_job_value(tokens, world, dt), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                "ms_per_step": dt * 1e3, "steps": e2e_steps, "api": "dkv_run_prefill_pass_host (pinned host buffers)"}
 
     B.dkv_destroy(ctx)
