@@ -23,18 +23,19 @@ namespace dkv {
 namespace tc {
 
 constexpr int kTileKeys = 128;
+constexpr int kMmaWarp2 = 18;
 constexpr int kStages = 4;                 // K tiles in flight
-constexpr int kThreads = 576;              // warp 0: TMA, warp 1: MMA, warps 2..17: softmax
+constexpr int kThreads = 608;              // warp 0: TMA, warps 1 and 18: MMA (even / odd tiles), warps 2..17: softmax
 constexpr int kSoftmaxThreads = 512;
-constexpr int kParts = 4;                  // softmax warps per TMEM lane quadrant
-constexpr int kMaxSegTiles = 8;            // sweep 2: tiles per pooled segment
+constexpr int kParts = 4;                  // softmax warps per TMEM lane quadrant: 2 tile groups x 2 column halves
+constexpr int kMaxSegTiles = 16;           // sweep 2: tiles per pooled segment
 constexpr int kStageCols = 256;            // TMEM columns per accumulator stage
 constexpr int kQTmemCol = 128;             // sweep 1 with one 128-row block: the queries sit in columns [128, 192)
 constexpr int kHalfBytes = 128 * 128;      // one 128-row x 64-column bf16 box
 constexpr int kQRegion = 2 * 2 * kHalfBytes;          // up to 256 rows x 128 columns
 constexpr int kKRegion = kStages * 2 * kHalfBytes;    // ring of 128 x 128 tiles
 constexpr int kMiscBytes = 1024 /*lse*/ + 3 * 256 * 8 /*merge*/;
-constexpr int kRawBytes = kParts * kMaxSegTiles * kTileKeys * 4;
+constexpr int kRawBytes = 2 * kMaxSegTiles * kTileKeys * 4;   // sweep 2: one partial-sum array per column half
 constexpr int kSmemBytes = 1024 /*align*/ + kQRegion + kKRegion + kMiscBytes + kRawBytes + 256 /*barriers*/;
 constexpr long long kWaitCycles = 4000000000ll;       // ~2 s: a wait that long is reported, not spun on
 
@@ -229,7 +230,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
   uint8_t* k_smem = smem + kQRegion;                   // [stage][half][128 rows][128 B]
   float* lse_s = reinterpret_cast<float*>(k_smem + kKRegion);          // [256] lse2 per window row (sweep 2)
   float2* merge_s = reinterpret_cast<float2*>(lse_s + 256);            // [3][256] partials of column parts 1..3 (sweep 1)
-  float* raw_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(lse_s) + kMiscBytes);   // [part][8 * 128]
+  float* raw_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(lse_s) + kMiscBytes);   // [half][kMaxSegTiles * 128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(raw_s) + kRawBytes);
   // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2], q_full
   __shared__ uint32_t tmem_base_s;
@@ -248,7 +249,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
   if (threadIdx.x == 0) {
     abort_s = 0;
     for (int s = 0; s < kStages; ++s) { mbar_init(FULL(s), 1); mbar_init(EMPTY(s), 1); }
-    for (int t = 0; t < 2; ++t) { mbar_init(TFULL(t), 1); mbar_init(TEMPTY(t), 16); }
+    for (int t = 0; t < 2; ++t) { mbar_init(TFULL(t), 1); mbar_init(TEMPTY(t), 8); }
     mbar_init(QFULL, 1);
     mbar_init(QTMEM, 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -277,10 +278,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
         Seg sg;
         while (it.next(sg)) {
           if (sg.new_head) {
-            if (tile > 0) {   // every MMA that read the previous queries must have finished
-              const int last = tile - 1;
+            // every MMA that read the previous queries must have finished: the last tile of either issuer
+            for (int last = tile - 1; last >= 0 && last >= tile - 2; --last)
               mbar_wait(EMPTY(last % kStages), (last / kStages) & 1, abort_flag, p.status, 101);
-            }
             if (!*abort_flag && !(p.mode == kStats && p.nmblk == 1)) {
               mbar_expect_tx(QFULL, (uint32_t)(p.nmblk * halves) * kHalfBytes);
               for (int h = 0; h < halves; ++h)
@@ -300,10 +300,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 1 || warp == kMmaWarp2) {
+    // ------------------------------------------------------------------ MMA issuers
+    // Two threads on different schedulers share the work: tile i belongs to issuer i & 1, which is also its
+    // accumulator stage.  One thread alone needs about as long to issue a tile's instructions as the
+    // tensor core needs to run them.
     if (lane == 0) {
+      const int which = warp == 1 ? 0 : 1;
       int tile = 0, nq = 0, nqt = 0;
+      bool q_wait = false;
       for (int jb = 0; jb < 2; ++jb) {
         const Params& p = jb ? job1 : job0;
         if (p.mode == kNone) continue;
@@ -312,11 +317,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
         SegIter it(p, blockIdx.x, gridDim.x);
         Seg sg;
         while (it.next(sg)) {
-          if (sg.new_head) {
-            if (q_tmem) { mbar_wait(QTMEM, nqt & 1, abort_flag, p.status, 108); ++nqt; tc_fence_after(); }
-            else { mbar_wait(QFULL, nq & 1, abort_flag, p.status, 103); ++nq; }
-          }
+          // the wait for a head's queries is taken at this issuer's first tile of the head (it may have none)
+          if (sg.new_head) { q_wait = true; if (q_tmem) ++nqt; else ++nq; }
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
+            if ((tile & 1) != which) continue;
+            if (q_wait) {
+              q_wait = false;
+              if (q_tmem) { mbar_wait(QTMEM, (nqt - 1) & 1, abort_flag, p.status, 108); tc_fence_after(); }
+              else mbar_wait(QFULL, (nq - 1) & 1, abort_flag, p.status, 103);
+            }
             const int s = tile % kStages, n = tile / kStages, t = tile & 1, nt = tile >> 1;
             mbar_wait(FULL(s), n & 1, abort_flag, p.status, 104);
             mbar_wait(TEMPTY(t), (nt & 1) ^ 1, abort_flag, p.status, 105);
@@ -351,7 +360,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
     }
   } else {
     // ------------------------------------------------------------------ softmax warps
-    const int part = (warp - 2) >> 2;          // which quarter of the accumulator columns
+    const int part = (warp - 2) >> 2;          // 0..3: group (tile parity) and half of the accumulator columns
+    const int grp = part >> 1, half = part & 1;
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
     const int row = quad * 32 + lane;          // TMEM lane = window row (sweep 1) or key within the tile (sweep 2)
     const int sid = threadIdx.x - 64;          // 0..511 among the softmax threads
@@ -387,45 +397,50 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
           float mx[2] = {-INFINITY, -INFINITY}, sum[2] = {0.f, 0.f};
           const int limit0 = p.P + (row % p.ws), limit1 = p.P + ((row + 128) % p.ws);
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
-            const int t = tile & 1, nt = tile >> 1;
+            if ((tile & 1) != grp) continue;                   // the other group's tile
+            const int t = grp, nt = tile >> 1;
             mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 106);
             tc_fence_after();
-            const uint32_t taddr = lane_addr + (uint32_t)(t * kStageCols + part * 32);
-            const int kb = sg.key0 + i * kTileKeys + part * 32;
-            const bool need_mask = kb + 31 > p.P;
+            const uint32_t taddr = lane_addr + (uint32_t)(t * kStageCols + half * 64);
+            const int kb0 = sg.key0 + i * kTileKeys + half * 64;
+            const bool need_mask = kb0 + 63 > p.P;
 #pragma unroll
             for (int mb = 0; mb < 2; ++mb) {
               if (mb >= p.nmblk) break;
-              float xv[32];
-              tc_ld32(taddr + mb * 128, xv);
-              tc_wait_ld();
-              if (mb + 1 == p.nmblk) {                         // last read of this stage: release it
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(TEMPTY(t));
-              }
-              if (need_mask) {
-                const int limit = mb ? limit1 : limit0;
 #pragma unroll
-                for (int e = 0; e < 32; ++e) if (kb + e > limit) xv[e] = -INFINITY;
-              }
-              float cm = fmax3(xv[0], xv[1], xv[2]);
+              for (int hh = 0; hh < 2; ++hh) {
+                float xv[32];
+                tc_ld32(taddr + mb * 128 + hh * 32, xv);
+                tc_wait_ld();
+                if (mb + 1 == p.nmblk && hh == 1) {              // last read of this stage: release it
+                  tc_fence_before();
+                  __syncwarp();
+                  if (lane == 0) mbar_arrive(TEMPTY(t));
+                }
+                if (need_mask) {
+                  const int limit = mb ? limit1 : limit0;
+                  const int kb = kb0 + hh * 32;
 #pragma unroll
-              for (int e = 3; e < 31; e += 2) cm = fmax3(cm, xv[e], xv[e + 1]);
-              cm = fmaxf(cm, xv[31]);
-              if (cm == -INFINITY) continue;
-              const float mnew = fmaxf(mx[mb], cm * p.scale2);
-              if (mnew > mx[mb]) { sum[mb] *= fast_exp2(mx[mb] - mnew); mx[mb] = mnew; }
-              float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-              const float neg = -mx[mb];
+                  for (int e = 0; e < 32; ++e) if (kb + e > limit) xv[e] = -INFINITY;
+                }
+                float cm = fmax3(xv[0], xv[1], xv[2]);
 #pragma unroll
-              for (int e = 0; e < 32; e += 4) {
-                s0 += fast_exp2(fmaf(xv[e], p.scale2, neg));
-                s1 += fast_exp2(fmaf(xv[e + 1], p.scale2, neg));
-                s2 += fast_exp2(fmaf(xv[e + 2], p.scale2, neg));
-                s3 += fast_exp2(fmaf(xv[e + 3], p.scale2, neg));
+                for (int e = 3; e < 31; e += 2) cm = fmax3(cm, xv[e], xv[e + 1]);
+                cm = fmaxf(cm, xv[31]);
+                if (cm == -INFINITY) continue;
+                const float mnew = fmaxf(mx[mb], cm * p.scale2);
+                if (mnew > mx[mb]) { sum[mb] *= fast_exp2(mx[mb] - mnew); mx[mb] = mnew; }
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                const float neg = -mx[mb];
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                  s0 += fast_exp2(fmaf(xv[e], p.scale2, neg));
+                  s1 += fast_exp2(fmaf(xv[e + 1], p.scale2, neg));
+                  s2 += fast_exp2(fmaf(xv[e + 2], p.scale2, neg));
+                  s3 += fast_exp2(fmaf(xv[e + 3], p.scale2, neg));
+                }
+                sum[mb] += (s0 + s1) + (s2 + s3);
               }
-              sum[mb] += (s0 + s1) + (s2 + s3);
             }
           }
           // merge the four column parts and publish this CTA's statistics for the head
@@ -476,35 +491,35 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
             lse_s[sid] = lse;
           }
           asm volatile("bar.sync 1, 512;" ::: "memory");
-          const int nchunk = p.nq16 >> 4;               // 16-column chunks; this warp takes part, part+4, ...
-          float* my_raw = raw_s + part * (kMaxSegTiles * kTileKeys);
+          const int nchunk = p.nq16 >> 4;               // 16-column chunks; this warp takes half, half+2, ...
+          float* my_raw = raw_s + half * (kMaxSegTiles * kTileKeys);
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
-            const int t = tile & 1, nt = tile >> 1;
+            if ((tile & 1) != grp) continue;                   // the other group's tile
+            const int t = grp, nt = tile >> 1;
             mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 107);
             tc_fence_after();
             const uint32_t taddr = lane_addr + (uint32_t)(t * kStageCols);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-            for (int jj = 0; jj < 2; ++jj) {                  // two 16-column chunks per round
-              const int c0 = part + 8 * jj, c1 = c0 + 4;
+            for (int jj = 0; jj < 4; ++jj) {                  // two 16-column chunks per round
+              const int c0 = half + 4 * jj, c1 = c0 + 2;
+              if (c0 >= nchunk) break;
               float x0[16], x1[16];
-              if (c0 < nchunk) tc_ld16(taddr + c0 * 16, x0);
+              tc_ld16(taddr + c0 * 16, x0);
               if (c1 < nchunk) tc_ld16(taddr + c1 * 16, x1);
               tc_wait_ld();
-              if (jj == 1 || part + 8 >= nchunk) {             // this warp's last read of the stage: release it
+              if (c0 + 4 >= nchunk) {                          // this warp's last read of the stage: release it
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(TEMPTY(t));
               }
-              if (c0 < nchunk) {
 #pragma unroll
-                for (int e = 0; e < 16; e += 4) {
-                  const float4 ls = *reinterpret_cast<const float4*>(&lse_s[c0 * 16 + e]);
-                  a0 += fast_exp2(fmaf(x0[e], p.scale2, -ls.x));
-                  a1 += fast_exp2(fmaf(x0[e + 1], p.scale2, -ls.y));
-                  a2 += fast_exp2(fmaf(x0[e + 2], p.scale2, -ls.z));
-                  a3 += fast_exp2(fmaf(x0[e + 3], p.scale2, -ls.w));
-                }
+              for (int e = 0; e < 16; e += 4) {
+                const float4 ls = *reinterpret_cast<const float4*>(&lse_s[c0 * 16 + e]);
+                a0 += fast_exp2(fmaf(x0[e], p.scale2, -ls.x));
+                a1 += fast_exp2(fmaf(x0[e + 1], p.scale2, -ls.y));
+                a2 += fast_exp2(fmaf(x0[e + 2], p.scale2, -ls.z));
+                a3 += fast_exp2(fmaf(x0[e + 3], p.scale2, -ls.w));
               }
               if (c1 < nchunk) {
 #pragma unroll
@@ -516,18 +531,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
                   a3 += fast_exp2(fmaf(x1[e + 3], p.scale2, -ls.w));
                 }
               }
-              if (part + 8 >= nchunk) break;                   // no second round for this warp
             }
             my_raw[i * kTileKeys + row] = (a0 + a1) + (a2 + a3);
           }
           asm volatile("bar.sync 1, 512;" ::: "memory");
-          // add up the four column parts in a fixed order; raw_s[x] then belongs to key key0 + x
-          for (int x = sid; x < sg.ntiles * kTileKeys; x += kSoftmaxThreads) {
-            float v = raw_s[x];
-#pragma unroll
-            for (int q = 1; q < kParts; ++q) v += raw_s[q * (kMaxSegTiles * kTileKeys) + x];
-            raw_s[x] = v;
-          }
+          // add up the two column halves in a fixed order; raw_s[x] then belongs to key key0 + x
+          for (int x = sid; x < sg.ntiles * kTileKeys; x += kSoftmaxThreads)
+            raw_s[x] += raw_s[kMaxSegTiles * kTileKeys + x];
           asm volatile("bar.sync 1, 512;" ::: "memory");
           // Eq. 2's pooling over this segment
           for (int o = sg.out0 + sid; o < sg.out1; o += kSoftmaxThreads) {
