@@ -45,8 +45,11 @@ struct dkv_ctx {
   // tensor-core scoring
   int n_sms, tc_grid, tc_slots;
   float2* d_tc_stats;   // [3][Bt*Hkv][tc_slots][256]: partial softmax statistics, three layers in rotation
+  cudaStream_t hi;      // scoring launches of dkv_run_prefill_pass: highest priority, so that a freed SM goes to a
+                        // waiting scoring CTA before the side streams' many short CTAs
+  cudaStream_t upd;     // budget updates (rebudget + shrink) of dkv_run_prefill_pass, off the select streams
   cudaStream_t side[2]; // side streams of dkv_run_prefill_pass (select / gather / rebudget / shrink), layers alternate
-  cudaEvent_t ev_fork, ev_join[2], ev_update, ev_scored[DKV_MAX_LAYERS], ev_selected[DKV_MAX_LAYERS];
+  cudaEvent_t ev_fork, ev_join[3], ev_update, ev_scored[DKV_MAX_LAYERS], ev_selected[DKV_MAX_LAYERS];
   // host state
   uint8_t scored[DKV_MAX_LAYERS], selected[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
   long long launches;
@@ -332,7 +335,10 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
   if (rc) return rc;
   DKV_CUDA(c, cudaEventRecord(c->ev_fork, st));
   for (int i = 0; i < 2; ++i) DKV_CUDA(c, cudaStreamWaitEvent(c->side[i], c->ev_fork, 0));
-  bool updated = false;
+  DKV_CUDA(c, cudaStreamWaitEvent(c->hi, c->ev_fork, 0));
+  DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_fork, 0));
+  cudaStream_t caller = st;
+  st = c->hi;
   for (int l = 0; l <= s.L; ++l) {
     const int sl = l < s.L ? l : -1, el = l - 1;
     if ((rc = launch_score(c, sl, sl >= 0 ? q[sl] : nullptr, sl >= 0 ? k[sl] : nullptr, el, el >= 0 ? q[el] : nullptr,
@@ -348,19 +354,23 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
     DKV_CUDA(c, cudaEventRecord(c->ev_selected[el], sd));
     const bool update = ((el + 1) % s.m == 0) || (el + 1 == s.L && s.L % s.m != 0);
     if (update) {
-      // needs every earlier layer selected and gathered (the other side stream) and the previous update
-      if (el >= 1) DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_selected[el - 1], 0));
-      if (updated) DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_update, 0));
-      if ((rc = do_rebudget(c, el + 1, nullptr, sd))) return rc;
-      if ((rc = do_shrink(c, 0, el + 1, kb, vb, sd))) return rc;
-      DKV_CUDA(c, cudaEventRecord(c->ev_update, sd));
-      updated = true;
+      // needs every earlier layer selected and gathered (both select streams, each in layer order); the
+      // previous update precedes it on the same stream.  Later layers' select and gather do not wait for it:
+      // an update changes the counts and buffers of the layers before it only.
+      DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_selected[el], 0));
+      if (el >= 1) DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_selected[el - 1], 0));
+      if ((rc = do_rebudget(c, el + 1, nullptr, c->upd))) return rc;
+      if ((rc = do_shrink(c, 0, el + 1, kb, vb, c->upd))) return rc;
     }
   }
   for (int i = 0; i < 2; ++i) {
     DKV_CUDA(c, cudaEventRecord(c->ev_join[i], c->side[i]));
-    DKV_CUDA(c, cudaStreamWaitEvent(st, c->ev_join[i], 0));
+    DKV_CUDA(c, cudaStreamWaitEvent(caller, c->ev_join[i], 0));
   }
+  DKV_CUDA(c, cudaEventRecord(c->ev_join[2], c->hi));
+  DKV_CUDA(c, cudaStreamWaitEvent(caller, c->ev_join[2], 0));
+  DKV_CUDA(c, cudaEventRecord(c->ev_update, c->upd));
+  DKV_CUDA(c, cudaStreamWaitEvent(caller, c->ev_update, 0));
   return DKV_OK;
 }
 
@@ -369,10 +379,10 @@ void free_all(dkv_ctx* c) {
   cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_rb_state); cudaFree(c->d_rb_above); cudaFree(c->d_rb_hist1);
   cudaFree(c->d_rb_above2); cudaFree(c->d_rb_hist2); cudaFree(c->d_head_hist); cudaFree(c->d_head_offs);
   cudaFree(c->d_cand); cudaFree(c->d_cand_n); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
-  for (int i = 0; i < 2; ++i) {
-    if (c->side[i]) cudaStreamDestroy(c->side[i]);
-    if (c->ev_join[i]) cudaEventDestroy(c->ev_join[i]);
-  }
+  for (int i = 0; i < 2; ++i) if (c->side[i]) cudaStreamDestroy(c->side[i]);
+  if (c->hi) cudaStreamDestroy(c->hi);
+  if (c->upd) cudaStreamDestroy(c->upd);
+  for (int i = 0; i < 3; ++i) if (c->ev_join[i]) cudaEventDestroy(c->ev_join[i]);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_update) cudaEventDestroy(c->ev_update);
   for (int l = 0; l < DKV_MAX_LAYERS; ++l) {
@@ -492,10 +502,14 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMalloc(&c->d_cand_n, sizeof(unsigned int) * s.Bt));
   TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * 3 * heads * c->tc_slots * 256));
   TRY(cudaFuncSetAttribute(tc::score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
-  for (int i = 0; i < 2; ++i) {
-    TRY(cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking));
-    TRY(cudaEventCreateWithFlags(&c->ev_join[i], cudaEventDisableTiming));
+  for (int i = 0; i < 2; ++i) TRY(cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking));
+  TRY(cudaStreamCreateWithFlags(&c->upd, cudaStreamNonBlocking));
+  {
+    int least = 0, greatest = 0;
+    TRY(cudaDeviceGetStreamPriorityRange(&least, &greatest));
+    TRY(cudaStreamCreateWithPriority(&c->hi, cudaStreamNonBlocking, greatest));
   }
+  for (int i = 0; i < 3; ++i) TRY(cudaEventCreateWithFlags(&c->ev_join[i], cudaEventDisableTiming));
   TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
   TRY(cudaEventCreateWithFlags(&c->ev_update, cudaEventDisableTiming));
   for (int l = 0; l < s.L; ++l) {
