@@ -31,6 +31,29 @@ METRIC = "prefix tokens/s through 32-layer KV compression at 32K ctx; HBM GB/s v
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "mistral32k"
 NOMINAL_HBM_GBS = 8000.0
+
+# DRAM traffic of one scoring launch (dram__bytes_read.sum + dram__bytes_write.sum), taken once with ncu on
+# the 4-layer cut of the mistral32k shape (same per-layer shape, so the figure needs no scaling; see
+# profiles/score_tc_kernel_mistral32k_4layers.md).  It holds for the kernel source it was measured on and for
+# that per-layer shape only: any other source hash or shape reports null.
+NCU_TRAFFIC = {
+    "kernel_sha256": "85381973396d8a7da2ee51dfdd984f103c650fe739b73766f4116878cae7d5d4",
+    "shape": (8, 128, 1, 32768, 32),          # Hkv, D, Bt, S, ws
+    "bytes_per_launch": 134_960_000 + 3_980_000,
+}
+
+
+def ncu_traffic(w):
+    import hashlib
+    src = os.path.join(ROOT, "paper_2412_14838_b200", "csrc", "score_tc.cuh")
+    try:
+        with open(src, "rb") as f:
+            sha = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    if sha != NCU_TRAFFIC["kernel_sha256"] or (w.Hkv, w.D, w.Bt, w.S, w.ws) != NCU_TRAFFIC["shape"]:
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"]
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -259,7 +282,7 @@ def run_gpu(args, w):
                 "achieved": achieved, "peak": peak, "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})",
                 "unit": "GB/s", "frac": achieved / peak,
                 "algorithmic_bytes_per_launch": k_bytes, "avg_launch_ms": score_launch_ms,
-                "traffic": None,
+                "traffic": ncu_traffic(w),
                 "whole_pass": {"algorithmic_bytes": w.algorithmic_bytes(),
                                "achieved_gbs": w.algorithmic_bytes() / (ms_per_step * 1e-3) / 1e9,
                                "frac_of_measured_peak": w.algorithmic_bytes() / (ms_per_step * 1e-3) / 1e9 / peak,
