@@ -189,7 +189,6 @@ bool make_job(dkv_ctx* c, int mode, int layer, const void* q, const void* k, flo
   p->status = c->d_status;
   p->stats_grid = c->tc_grid;
   p->mode = mode;
-  p->q_ptr = static_cast<const uint16_t*>(q);
   p->idesc = mode == tc::kStats ? make_idesc(128, 128) : make_idesc(128, p->nq16);
   return true;
 }
@@ -766,7 +765,6 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   p.scores = scores_out; p.copy_out = nullptr;
   p.status = reinterpret_cast<int*>(su.ptr);
   p.stats_grid = grid;
-  p.q_ptr = static_cast<const uint16_t*>(q_win);
   p.mode = tc::kStats;
   p.idesc = make_idesc(128, 128);
   tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, qm, km, p, none);

@@ -8,13 +8,13 @@
 //                     2^(logit - lse_row) over the rows of its own key, which is the token's score
 //                     with no cross-thread reduction; the CTA then max-pools its key range.
 // Both sweeps share one pipeline: a TMA producer warp streams 128-key tiles of K (bf16, 128-byte
-// swizzle) through a shared-memory ring, one thread issues tcgen05.mma into double-buffered TMEM
-// accumulators, and sixteen warps read the accumulators back with tcgen05.ld (four warps per TMEM
-// lane quadrant, each taking a quarter of the columns).
+// swizzle) through a shared-memory ring; two threads in different warps issue tcgen05.mma (tile i goes to
+// issuer i mod 2) into TMEM accumulator stages; sixteen warps read the accumulators back with tcgen05.ld
+// in two groups that alternate tiles, each warp one TMEM lane quadrant x half the columns.
 // Work is split evenly: the flattened (head, key tile) space for sweep 1 and the flattened
 // (head, prefix position) space for sweep 2 are cut into one contiguous slice per CTA.
-// One launch runs up to two jobs back to back through the same pipeline (sweep 1 of one layer, then
-// sweep 2 of the layer before it), so the fixed cost of a launch is paid once per layer.
+// One launch runs up to two jobs back to back through the same pipeline (sweep 2 of one layer, then
+// sweep 1 of the next), so the fixed cost of a launch is paid once per layer.
 #pragma once
 #include <cuda.h>
 #include "common.cuh"
@@ -29,8 +29,8 @@ constexpr int kThreads = 608;              // warp 0: TMA, warps 1 and 18: MMA (
 constexpr int kSoftmaxThreads = 512;
 constexpr int kParts = 4;                  // softmax warps per TMEM lane quadrant: 2 tile groups x 2 column halves
 constexpr int kMaxSegTiles = 16;           // sweep 2: tiles per pooled segment
-constexpr int kStageCols = 256;            // TMEM columns per accumulator stage
-constexpr int kQTmemCol = 128;             // sweep 1 with one 128-row block: the queries sit in columns [128, 192)
+// TMEM accumulator stages: four of 128 columns when the window rows fit one 128-row block (ws*G <= 128),
+// else two of 256.  A softmax group then always has a second accumulator being filled while it reads one.
 constexpr int kHalfBytes = 128 * 128;      // one 128-row x 64-column bf16 box
 constexpr int kQRegion = 2 * 2 * kHalfBytes;          // up to 256 rows x 128 columns
 constexpr int kKRegion = kStages * 2 * kHalfBytes;    // ring of 128 x 128 tiles
@@ -56,7 +56,6 @@ struct Params {
   int* status;             // device status words; [0] = first error
   int stats_grid;          // CTAs of the launch that ran sweep 1 for this layer
   int mode;                // kNone: nothing to do
-  const uint16_t* q_ptr;   // window queries bf16 [heads][M][D] (sweep 1 with ws*G <= 128 keeps them in TMEM)
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -112,24 +111,6 @@ __device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 // A operand from tensor memory (128 rows = lanes, 16-bit elements packed two per column), B from shared memory.
-__device__ __forceinline__ void tc_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
-        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
-        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
   uint32_t r[16];
   asm volatile(
@@ -239,9 +220,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
   auto FULL = [&](int s) { return bar0 + 8u * s; };
   auto EMPTY = [&](int s) { return bar0 + 8u * (kStages + s); };
   auto TFULL = [&](int t) { return bar0 + 8u * (2 * kStages + t); };
-  auto TEMPTY = [&](int t) { return bar0 + 8u * (2 * kStages + 2 + t); };
-  const uint32_t QFULL = bar0 + 8u * (2 * kStages + 4);
-  const uint32_t QTMEM = bar0 + 8u * (2 * kStages + 5);      // queries stored to tensor memory (sweep 1)
+  auto TEMPTY = [&](int t) { return bar0 + 8u * (2 * kStages + 4 + t); };
+  const uint32_t QFULL = bar0 + 8u * (2 * kStages + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &abort_s;
@@ -249,9 +229,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
   if (threadIdx.x == 0) {
     abort_s = 0;
     for (int s = 0; s < kStages; ++s) { mbar_init(FULL(s), 1); mbar_init(EMPTY(s), 1); }
-    for (int t = 0; t < 2; ++t) { mbar_init(TFULL(t), 1); mbar_init(TEMPTY(t), 8); }
+    for (int t = 0; t < 4; ++t) { mbar_init(TFULL(t), 1); mbar_init(TEMPTY(t), 8); }
     mbar_init(QFULL, 1);
-    mbar_init(QTMEM, 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -281,7 +260,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
             // every MMA that read the previous queries must have finished: the last tile of either issuer
             for (int last = tile - 1; last >= 0 && last >= tile - 2; --last)
               mbar_wait(EMPTY(last % kStages), (last / kStages) & 1, abort_flag, p.status, 101);
-            if (!*abort_flag && !(p.mode == kStats && p.nmblk == 1)) {
+            if (!*abort_flag) {
               mbar_expect_tx(QFULL, (uint32_t)(p.nmblk * halves) * kHalfBytes);
               for (int h = 0; h < halves; ++h)
                 for (int mb = 0; mb < p.nmblk; ++mb)
@@ -307,38 +286,30 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
     // tensor core needs to run them.
     if (lane == 0) {
       const int which = warp == 1 ? 0 : 1;
-      int tile = 0, nq = 0, nqt = 0;
+      int tile = 0, nq = 0;
       bool q_wait = false;
       for (int jb = 0; jb < 2; ++jb) {
         const Params& p = jb ? job1 : job0;
         if (p.mode == kNone) continue;
         const int ksteps = p.D / 16;
-        const bool q_tmem = p.mode == kStats && p.nmblk == 1;
+        const int tmask = p.nmblk == 1 ? 3 : 1, tshift = p.nmblk == 1 ? 2 : 1, scols = p.nmblk == 1 ? 128 : 256;
         SegIter it(p, blockIdx.x, gridDim.x);
         Seg sg;
         while (it.next(sg)) {
           // the wait for a head's queries is taken at this issuer's first tile of the head (it may have none)
-          if (sg.new_head) { q_wait = true; if (q_tmem) ++nqt; else ++nq; }
+          if (sg.new_head) { q_wait = true; ++nq; }
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
             if ((tile & 1) != which) continue;
             if (q_wait) {
               q_wait = false;
-              if (q_tmem) { mbar_wait(QTMEM, (nqt - 1) & 1, abort_flag, p.status, 108); tc_fence_after(); }
-              else mbar_wait(QFULL, (nq - 1) & 1, abort_flag, p.status, 103);
+              mbar_wait(QFULL, (nq - 1) & 1, abort_flag, p.status, 103);
             }
-            const int s = tile % kStages, n = tile / kStages, t = tile & 1, nt = tile >> 1;
+            const int s = tile % kStages, n = tile / kStages, t = tile & tmask, nt = tile >> tshift;
             mbar_wait(FULL(s), n & 1, abort_flag, p.status, 104);
             mbar_wait(TEMPTY(t), (nt & 1) ^ 1, abort_flag, p.status, 105);
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(t * kStageCols);
-            if (q_tmem) {
-              // the queries never change within a head: read them from tensor memory, so that shared memory
-              // only has to feed the key tile to the tensor core
-              for (int ks = 0; ks < ksteps; ++ks) {
-                const uint64_t b = smem_desc(smem_u32(k_smem + (s * 2 + (ks >> 2)) * kHalfBytes) + (ks & 3) * 32);
-                tc_mma_ts(d_tmem, tmem_base + kQTmemCol + ks * 8, b, p.idesc, ks > 0);
-              }
-            } else if (p.mode == kStats) {
+            const uint32_t d_tmem = tmem_base + (uint32_t)(t * scols);
+            if (p.mode == kStats) {
               for (int mb = 0; mb < p.nmblk; ++mb)
                 for (int ks = 0; ks < ksteps; ++ks) {
                   const uint64_t a = smem_desc(smem_u32(q_smem + (ks >> 2) * (2 * kHalfBytes) + mb * kHalfBytes) + (ks & 3) * 32);
@@ -372,36 +343,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
       if (p.mode == kNone) continue;
       SegIter it(p, blockIdx.x, gridDim.x);
       Seg sg;
+      const int tmask = p.nmblk == 1 ? 3 : 1, tshift = p.nmblk == 1 ? 2 : 1, scols = p.nmblk == 1 ? 128 : 256;
       while (it.next(sg)) {
         if (p.mode == kStats) {
           // ------------------------------------------------------------ sweep 1: (max, sum) per window row
-          if (sg.new_head && p.nmblk == 1 && part == 0) {
-            // this warp has consumed every earlier tile, so every MMA that read the old queries is done:
-            // store this head's queries, row = TMEM lane, two bf16 per 32-bit column
-            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(p.q_ptr + ((size_t)sg.bh * p.M + row) * p.D);
-            for (int c = 0; c < p.D / 2; c += 32) {
-              uint32_t qv[32];
-#pragma unroll
-              for (int e = 0; e < 32; e += 4) {
-                uint4 w = make_uint4(0, 0, 0, 0);
-                if (row < p.M) w = *reinterpret_cast<const uint4*>(qrow + c + e);
-                qv[e] = w.x; qv[e + 1] = w.y; qv[e + 2] = w.z; qv[e + 3] = w.w;
-              }
-              tc_st32(lane_addr + kQTmemCol + c, qv);
-            }
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(QTMEM);
-          }
           float mx[2] = {-INFINITY, -INFINITY}, sum[2] = {0.f, 0.f};
           const int limit0 = p.P + (row % p.ws), limit1 = p.P + ((row + 128) % p.ws);
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
             if ((tile & 1) != grp) continue;                   // the other group's tile
-            const int t = grp, nt = tile >> 1;
+            const int t = tile & tmask, nt = tile >> tshift;
             mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 106);
             tc_fence_after();
-            const uint32_t taddr = lane_addr + (uint32_t)(t * kStageCols + half * 64);
+            const uint32_t taddr = lane_addr + (uint32_t)(t * scols + half * 64);
             const int kb0 = sg.key0 + i * kTileKeys + half * 64;
             const bool need_mask = kb0 + 63 > p.P;
 #pragma unroll
@@ -495,10 +448,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
           float* my_raw = raw_s + half * (kMaxSegTiles * kTileKeys);
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
             if ((tile & 1) != grp) continue;                   // the other group's tile
-            const int t = grp, nt = tile >> 1;
+            const int t = tile & tmask, nt = tile >> tshift;
             mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 107);
             tc_fence_after();
-            const uint32_t taddr = lane_addr + (uint32_t)(t * kStageCols);
+            const uint32_t taddr = lane_addr + (uint32_t)(t * scols);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
             for (int jj = 0; jj < 4; ++jj) {                  // two 16-column chunks per round
