@@ -453,6 +453,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
             tc_fence_after();
             const uint32_t taddr = lane_addr + (uint32_t)(t * scols);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            if (half >= nchunk) {                              // a single chunk (ws*G <= 16): nothing for this warp to read
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(TEMPTY(t));
+            }
 #pragma unroll
             for (int jj = 0; jj < 4; ++jj) {                  // two 16-column chunks per round
               const int c0 = half + 4 * jj, c1 = c0 + 2;
