@@ -55,3 +55,17 @@ def test_reference_arm_other_ranks_do_nothing():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1"],
                        env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_ncu_traffic_is_tied_to_kernel_source_and_shape(monkeypatch):
+    """The stored DRAM-traffic figures are reported only for the kernel source and per-layer shape they were
+    measured on; anything else must give null rather than a stale number."""
+    import bench
+    from paper_2412_14838_b200 import synth
+    w = synth.WORKLOADS["mistral32k"]
+    got = bench.ncu_traffic(w)
+    if got is not None:                       # the source is the measured one
+        assert got["cold_bytes_per_launch"] >= got["live_bytes_per_launch"] >= w.k_bytes_per_layer()
+    assert bench.ncu_traffic(synth.WORKLOADS["tiny"]) is None
+    monkeypatch.setitem(bench.NCU_TRAFFIC, "kernel_sha256", "0" * 64)
+    assert bench.ncu_traffic(w) is None
