@@ -29,8 +29,7 @@ struct dkv_ctx {
   int* d_count;         // [Bt][L] budget of each layer
   int* d_held;          // [Bt][L] rows the layer's buffers hold
   int* d_dbg;           // 3 x [Bt][L] : cnt, Z, Z' of the last update
-  unsigned int* d_head_hist;  // [L][Bt][Hkv][2048] first-digit histogram of every head's scores
-  unsigned int* d_head_offs;  // [L][Bt][Hkv][2048] its ascending exclusive offsets
+  unsigned int* d_layer_hist; // [L][Bt][2048] first-digit histogram of every layer's scores (all heads of a sample)
   uint2* d_cand;              // [Bt][L*Hkv*P] (score bits, layer) of the scores in the global top-K's first bucket
   unsigned int* d_cand_n;     // [Bt]
   RbState* d_rb_state;        // [Bt]
@@ -235,14 +234,14 @@ int do_select(dkv_ctx* c, int layer, int* sorted_out, int* rank_out, cudaStream_
   ProfScope ps(c, DKV_STEP_SELECT, 1, st);
   const float* sc = c->d_scores + (size_t)layer * layer_scores(s);
   int* idx = c->d_idx + (size_t)layer * layer_idx(s);
-  unsigned int* hh = c->d_head_hist + (size_t)layer * heads * kBins;
-  unsigned int* ho = c->d_head_offs + (size_t)layer * heads * kBins;
+  unsigned int* lh = c->d_layer_hist + (size_t)layer * s.Bt * kBins;
+  DKV_CUDA(c, cudaMemsetAsync(lh, 0, sizeof(unsigned int) * s.Bt * kBins, st));
   if (c->sel_reg)
     select_topk_kernel<true><<<(unsigned)heads, kSelThreads, c->sel_smem, st>>>(
-        sc, idx, sorted_out, rank_out, hh, ho, s.P, s.Blc, c->sort_n, c->d_count, s.Hkv, s.L, layer);
+        sc, idx, sorted_out, rank_out, lh, s.P, s.Blc, c->sort_n, c->d_count, s.Hkv, s.L, layer);
   else
     select_topk_kernel<false><<<(unsigned)heads, kSelThreads, c->sel_smem, st>>>(
-        sc, idx, sorted_out, rank_out, hh, ho, s.P, s.Blc, c->sort_n, c->d_count, s.Hkv, s.L, layer);
+        sc, idx, sorted_out, rank_out, lh, s.P, s.Blc, c->sort_n, c->d_count, s.Hkv, s.L, layer);
   DKV_LAUNCHED(c);
   c->selected[layer] = 1;
   c->gathered[layer] = c->stale[layer] = 0;
@@ -257,7 +256,7 @@ int do_rebudget(dkv_ctx* c, int l, int* counts_out, cudaStream_t st) {
   if (k > pop) k = pop;
   ProfScope ps(c, DKV_STEP_REBUDGET, 4, st);
   const size_t per_layer = (size_t)s.Hkv * s.P, cand_stride = (size_t)s.L * per_layer;
-  rb_locate_kernel<<<s.Bt, 1024, 0, st>>>(c->d_head_hist, c->d_head_offs, c->d_rb_state, c->d_rb_above, c->d_rb_hist1,
+  rb_locate_kernel<<<s.Bt, 1024, 0, st>>>(c->d_layer_hist, c->d_rb_state, c->d_rb_above, c->d_rb_hist1,
                                          c->d_rb_above2, c->d_rb_hist2, c->d_cand_n, s.Bt, s.Hkv, s.L, l, s.P, k);
   DKV_LAUNCHED(c);
   int slices = (int)((per_layer + (size_t)kRbThreads * 16 - 1) / ((size_t)kRbThreads * 16));
@@ -265,7 +264,7 @@ int do_rebudget(dkv_ctx* c, int l, int* counts_out, cudaStream_t st) {
   rb_refine1_kernel<<<dim3(slices, l, s.Bt), kRbThreads, 0, st>>>(c->d_scores, c->d_rb_state, c->d_rb_hist1, c->d_cand,
                                                                  c->d_cand_n, s.Bt, per_layer, cand_stride);
   DKV_LAUNCHED(c);
-  rb_refine2_kernel<<<dim3(64, s.Bt), kRbThreads, 0, st>>>(c->d_cand, c->d_cand_n, c->d_rb_state, c->d_rb_hist1,
+  rb_refine2_kernel<<<dim3(256, s.Bt), kRbThreads, 0, st>>>(c->d_cand, c->d_cand_n, c->d_rb_state, c->d_rb_hist1,
                                                           c->d_rb_above2, c->d_rb_hist2, s.L, cand_stride);
   DKV_LAUNCHED(c);
   const size_t bl = (size_t)s.Bt * s.L;
@@ -376,7 +375,7 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
 void free_all(dkv_ctx* c) {
   cudaFree(c->d_scores); cudaFree(c->d_idx); cudaFree(c->d_count);
   cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_rb_state); cudaFree(c->d_rb_above); cudaFree(c->d_rb_hist1);
-  cudaFree(c->d_rb_above2); cudaFree(c->d_rb_hist2); cudaFree(c->d_head_hist); cudaFree(c->d_head_offs);
+  cudaFree(c->d_rb_above2); cudaFree(c->d_rb_hist2); cudaFree(c->d_layer_hist);
   cudaFree(c->d_cand); cudaFree(c->d_cand_n); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
   for (int i = 0; i < 2; ++i) if (c->side[i]) cudaStreamDestroy(c->side[i]);
   if (c->hi) cudaStreamDestroy(c->hi);
@@ -495,8 +494,7 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMalloc(&c->d_rb_above2, sizeof(unsigned int) * bl));
   TRY(cudaMalloc(&c->d_rb_hist1, sizeof(unsigned int) * s.Bt * kBins));
   TRY(cudaMalloc(&c->d_rb_hist2, sizeof(unsigned int) * bl * 1024));
-  TRY(cudaMalloc(&c->d_head_hist, sizeof(unsigned int) * s.L * heads * kBins));
-  TRY(cudaMalloc(&c->d_head_offs, sizeof(unsigned int) * s.L * heads * kBins));
+  TRY(cudaMalloc(&c->d_layer_hist, sizeof(unsigned int) * s.L * s.Bt * kBins));
   TRY(cudaMalloc(&c->d_cand, sizeof(uint2) * s.L * layer_scores(s)));
   TRY(cudaMalloc(&c->d_cand_n, sizeof(unsigned int) * s.Bt));
   TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * 3 * heads * c->tc_slots * 256));

@@ -1,10 +1,10 @@
 // Update_Buffer_Length (Eq. 4-6) on the device: the K-th largest of all scores of the layers processed
 // so far, the number of top-K hits per layer, then the integer budget arithmetic.
 //
-// Only per-layer counts leave the selection.  Every head's scores were histogrammed by their first
+// Only per-layer counts leave the selection.  Every layer's scores were histogrammed by their first
 // 11-bit digit when the layer was selected (select.cuh), so:
-//   rb_locate   adds up the per-head histograms of layers [0, l), finds the digit b* that holds the K-th
-//               largest score, and reads each layer's count of scores above b* off the offsets;
+//   rb_locate   adds up the histograms of layers [0, l), finds the digit b* that holds the K-th
+//               largest score, and counts each layer's scores above b* from its histogram;
 //   rb_refine1  streams the history once, copies the scores whose first digit is b* (with their layer)
 //               into a candidate list and histograms their next 11 bits;
 //   rb_refine2  counts, per layer, the candidates above the second digit and histograms the last
@@ -27,33 +27,26 @@ struct RbState {          // per sample
 };
 
 // One CTA of 1024 threads per sample.
-// head_hist/head_offs: [L][Bt][Hkv][2048].  above: [Bt][L] scores above bucket b* per layer.
+// layer_hist: [L][Bt][2048].  above: [Bt][L] scores above bucket b* per layer.
 // hist1: [Bt][2048], above2: [Bt][L], hist2: [Bt][L][1024], cand_n: [Bt] are cleared here for the refine kernels.
 __global__ void __launch_bounds__(1024)
-rb_locate_kernel(const unsigned int* __restrict__ head_hist, const unsigned int* __restrict__ head_offs,
-                 RbState* __restrict__ state, unsigned int* __restrict__ above, unsigned int* __restrict__ hist1,
-                 unsigned int* __restrict__ above2, unsigned int* __restrict__ hist2, unsigned int* __restrict__ cand_n,
-                 int Bt, int Hkv, int L, int l, int P, long long k) {
+rb_locate_kernel(const unsigned int* __restrict__ layer_hist, RbState* __restrict__ state,
+                 unsigned int* __restrict__ above, unsigned int* __restrict__ hist1, unsigned int* __restrict__ above2,
+                 unsigned int* __restrict__ hist2, unsigned int* __restrict__ cand_n, int Bt, int Hkv, int L, int l, int P,
+                 long long k) {
   __shared__ unsigned int hist[kBins];
   __shared__ int sm_scan[33];
   __shared__ int found[2];
-  const int b = blockIdx.x, tid = threadIdx.x;
-  for (int bin = tid; bin < kBins; bin += 1024) { hist[bin] = 0; hist1[(size_t)b * kBins + bin] = 0; }
-  __syncthreads();
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   {
-    // four groups of 256 threads walk the (layer, head) list in parallel, eight digits per thread
-    const int g = tid >> 8, c = tid & 255;
-    uint4 a0 = make_uint4(0, 0, 0, 0), a1 = make_uint4(0, 0, 0, 0);
-    for (int ih = g; ih < l * Hkv; ih += 4) {
-      const int i = ih / Hkv, h = ih % Hkv;
-      const uint4* src = reinterpret_cast<const uint4*>(head_hist + (((size_t)i * Bt + b) * Hkv + h) * kBins) + 2 * c;
-      const uint4 x = src[0], y = src[1];
-      a0.x += x.x; a0.y += x.y; a0.z += x.z; a0.w += x.w;
-      a1.x += y.x; a1.y += y.y; a1.z += y.z; a1.w += y.w;
+    // two digits per thread, summed over the layers (consecutive threads read consecutive words)
+    uint2 a = make_uint2(0, 0);
+    for (int i = 0; i < l; ++i) {
+      const uint2 x = reinterpret_cast<const uint2*>(layer_hist + ((size_t)i * Bt + b) * kBins)[tid];
+      a.x += x.x; a.y += x.y;
     }
-    unsigned int* hb = hist + 8 * c;
-    atomicAdd(hb + 0, a0.x); atomicAdd(hb + 1, a0.y); atomicAdd(hb + 2, a0.z); atomicAdd(hb + 3, a0.w);
-    atomicAdd(hb + 4, a1.x); atomicAdd(hb + 5, a1.y); atomicAdd(hb + 6, a1.z); atomicAdd(hb + 7, a1.w);
+    hist[2 * tid] = a.x; hist[2 * tid + 1] = a.y;
+    hist1[(size_t)b * kBins + 2 * tid] = 0; hist1[(size_t)b * kBins + 2 * tid + 1] = 0;
   }
   if (tid == 0) cand_n[b] = 0;
   for (int e = tid; e < L; e += 1024) above2[b * L + e] = 0;
@@ -63,13 +56,14 @@ rb_locate_kernel(const unsigned int* __restrict__ head_hist, const unsigned int*
   find_digit(hist, kBins, (int)total, (int)k, sm_scan, found, nullptr);
   const int d = found[0];
   if (tid == 0) { RbState st; st.bstar = d; st.need1 = found[1]; st.cand = (int)hist[d]; st.pad = 0; state[b] = st; }
-  for (int i = tid; i < l; i += 1024) {
+  // one warp per layer: the layer's scores in the digits above b*
+  for (int i = warp; i < l; i += 32) {
+    const unsigned int* lh = layer_hist + ((size_t)i * Bt + b) * kBins;
     unsigned int a = 0;
-    for (int h = 0; h < Hkv; ++h) {
-      const size_t at = (((size_t)i * Bt + b) * Hkv + h) * kBins + d;
-      a += (unsigned int)P - head_offs[at] - head_hist[at];
-    }
-    above[b * L + i] = a;
+    for (int bin = d + 1 + lane; bin < kBins; bin += 32) a += lh[bin];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
+    if (lane == 0) above[b * L + i] = a;
   }
 }
 
@@ -182,28 +176,47 @@ rb_budget_kernel(const RbState* __restrict__ state, const unsigned int* __restri
     }
   }
   __syncthreads();
-  if (tid == 0) {
-    long long cmax = 0;
-    for (int i = 0; i < l; ++i) {
-      const long long take = ties < s_eq[i] ? ties : s_eq[i];
-      ties -= take;
-      s_gt[i] += take;                        // = cnt_i
-      dbg_cnt[b * L + i] = (int)s_gt[i];
-      cmax = s_gt[i] > cmax ? s_gt[i] : cmax;
+  // Eq. 5-6 with one thread per layer (warp 0; layers lane, lane + 32, ...): the ties go to the lowest layers
+  // first, i.e. layer i takes min(eq_i, ties - sum of eq below i).
+  if (warp == 0) {
+    long long carry = 0, cmax = 0;
+    for (int i0 = 0; i0 < l; i0 += 32) {
+      const int i = i0 + lane;
+      const long long eq = i < l ? s_eq[i] : 0;
+      long long incl = eq;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const long long y = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += y; }
+      const long long before = carry + incl - eq;
+      long long take = ties - before;
+      take = take < 0 ? 0 : (take < eq ? take : eq);
+      if (i < l) {
+        s_gt[i] += take;                      // = cnt_i
+        dbg_cnt[b * L + i] = (int)s_gt[i];
+        cmax = s_gt[i] > cmax ? s_gt[i] : cmax;
+      }
+      carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { const long long y = __shfl_xor_sync(0xFFFFFFFFu, cmax, o); cmax = y > cmax ? y : cmax; }
     if (cmax <= 0) cmax = 1;
     long long sumz = 0;
-    for (int i = 0; i < l; ++i) { s_eq[i] = ((long long)Bl * s_gt[i]) / cmax; dbg_z[b * L + i] = (int)s_eq[i]; sumz += s_eq[i]; }
+    for (int i = lane; i < l; i += 32) {
+      s_eq[i] = ((long long)Bl * s_gt[i]) / cmax;             // Z_i
+      dbg_z[b * L + i] = (int)s_eq[i];
+      sumz += s_eq[i];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sumz += __shfl_xor_sync(0xFFFFFFFFu, sumz, o);
     if (sumz <= 0) sumz = 1;
     const long long B = (long long)N * L;
-    for (int i = 0; i < l; ++i) {
-      const long long zp = (s_eq[i] * B) / sumz;
+    for (int i = lane; i < l; i += 32) {
+      const long long zp = (s_eq[i] * B) / sumz;              // Z'_i
       const int zpi = zp > 0x7FFFFFFF ? 0x7FFFFFFF : (int)zp;
       dbg_zp[b * L + i] = zpi;
       const int c = count[b * L + i];
       count[b * L + i] = c < zpi ? c : zpi;
     }
-    for (int i = l; i < L; ++i) { dbg_cnt[b * L + i] = 0; dbg_z[b * L + i] = 0; dbg_zp[b * L + i] = 0; }
+    for (int i = l + lane; i < L; i += 32) { dbg_cnt[b * L + i] = 0; dbg_z[b * L + i] = 0; dbg_zp[b * L + i] = 0; }
   }
   __syncthreads();
   if (counts_out) for (int i = tid; i < L; i += 1024) counts_out[b * L + i] = count[b * L + i];

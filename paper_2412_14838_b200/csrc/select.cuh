@@ -122,14 +122,15 @@ __device__ __forceinline__ void bitonic_sort(unsigned long long* keys, int sort_
 // scores: [Bt*Hkv][P] of one layer.
 // idx: [Bt*Hkv][keep] kept positions in buffer order = (score descending, position ascending).
 // sorted_out (optional): the same positions ascending; rank_out (optional): rank of each of those.
-// head_hist, head_offs: [Bt*Hkv][2048] first-digit counts of the head and their ascending exclusive offsets.
+// layer_hist: [Bt][2048] first-digit counts of the layer's scores, all heads of a sample added up (zeroed by
+// the host before the launch); the rebudget works from these.
 // Also records count[b][layer] = keep.
 // Every warp owns a run of 32*chunk consecutive positions; lane j holds positions run + 32*e + j.
 // Dynamic shared memory: 8*sort_n bytes, then 4*keep bytes.
 template <bool REG>
 __global__ void __launch_bounds__(kSelThreads)
 select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int* __restrict__ sorted_out,
-                   int* __restrict__ rank_out, unsigned int* __restrict__ head_hist, unsigned int* __restrict__ head_offs,
+                   int* __restrict__ rank_out, unsigned int* __restrict__ layer_hist,
                    int P, int keep, int sort_n, int* __restrict__ count, int Hkv, int L, int layer) {
   extern __shared__ __align__(16) unsigned char dyn[];
   __shared__ unsigned int hist[kBins];
@@ -165,10 +166,10 @@ select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int*
   DKV_SEL_FOR(e) agg_bump(hist, val(e) >> 21, DKV_SEL_OK(e));
   __syncthreads();
   {
-    unsigned int* gh = head_hist + (size_t)blockIdx.x * kBins;
-    for (int i = tid; i < kBins; i += kSelThreads) gh[i] = hist[i];
+    unsigned int* gh = layer_hist + (size_t)(blockIdx.x / Hkv) * kBins;
+    for (int i = tid; i < kBins; i += kSelThreads) { const unsigned int c = hist[i]; if (c) atomicAdd(&gh[i], c); }
   }
-  find_digit(hist, kBins, P, keep, sm_scan, found, head_offs + (size_t)blockIdx.x * kBins);
+  find_digit(hist, kBins, P, keep, sm_scan, found, nullptr);
   uint32_t prefix = ((uint32_t)found[0]) << 21, mask = 2047u << 21;
   int need = found[1], total = (int)hist[found[0]];
   __syncthreads();
