@@ -17,6 +17,10 @@ prefix tokens, ``N = wt - ws``, ``B^l`` = ``Bl`` per-layer maximum, ``m`` update
 * ``shrink_rows``          Algorithm 1's truncation of every preceding layer's buffer.
 * ``run_prefill_pass``     Algorithm 1's loop over layers.
 
+Alternative readings, off by default, selectable per call: the window MEAN instead of the sum, an
+average pool (``avg_pool_same``), the pro-rata budget ``B = N * l`` at an intermediate update, and
+min-max normalisation of the layer counts.
+
 Readings taken where the paper is silent or inconsistent (each is listed in the design
 notes): window reduction is a SUM over the ``ws`` window rows and the ``G`` query heads of a KV
 head (the mean differs by a constant factor and selects the same tokens); logits are scaled by
@@ -76,7 +80,27 @@ def max_pool_same(x: np.ndarray, kernel: int) -> np.ndarray:
     return out
 
 
-def window_scores(q_win: np.ndarray, k: np.ndarray, ws: int, pool: int) -> Dict[str, np.ndarray]:
+def avg_pool_same(x: np.ndarray, kernel: int) -> np.ndarray:
+    """Stride-1 average pool of odd width along the last axis: the mean over the neighbours that exist
+    (an alternative reading of the paper's unspecified "pooling"; the default is the max-pool above)."""
+    if kernel % 2 != 1 or kernel < 1:
+        raise ValueError("pool kernel must be odd and >= 1")
+    half = kernel // 2
+    n = x.shape[-1]
+    tot = x.copy()
+    cnt = np.ones(n, dtype=np.float64)
+    for off in range(1, half + 1):
+        if off >= n:
+            break
+        tot[..., :-off] += x[..., off:]
+        tot[..., off:] += x[..., :-off]
+        cnt[:-off] += 1
+        cnt[off:] += 1
+    return tot / cnt
+
+
+def window_scores(q_win: np.ndarray, k: np.ndarray, ws: int, pool: int, *, pool_kind: int = 0,
+                  window_mean: bool = False) -> Dict[str, np.ndarray]:
     """Eq. 2 / Algorithm 1's scoring line for one layer.
 
     ``q_win`` [Bt, Hq, ws, D] and ``k`` [Bt, Hkv, S, D] in float64 (exactly widened bf16).
@@ -86,6 +110,9 @@ def window_scores(q_win: np.ndarray, k: np.ndarray, ws: int, pool: int) -> Dict[
     Returns ``score`` [Bt, Hkv, P] (pooled), ``raw`` [Bt, Hkv, P] (un-pooled) and ``window_mass``
     [Bt, Hkv] (probability that fell on the window's own columns), so that
     ``raw.sum(-1) + window_mass == ws * G`` can be checked.
+
+    Variant readings: ``window_mean`` takes Algorithm 1's ``.mean`` over the window rows (and the group)
+    instead of the sum, i.e. divides ``raw`` by ``ws * G``; ``pool_kind = 1`` pools with the average.
     """
     Bt, Hq, ws_, D = q_win.shape
     _, Hkv, S, _ = k.shape
@@ -99,7 +126,10 @@ def window_scores(q_win: np.ndarray, k: np.ndarray, ws: int, pool: int) -> Dict[
                 A = softmax_rows_causal(q_win[b, h * G + g], k[b, h], P)   # [ws, S]
                 raw[b, h] += A[:, :P].sum(axis=0)
                 wmass[b, h] += A[:, P:].sum()
-    return {"score": max_pool_same(raw, pool), "raw": raw, "window_mass": wmass}
+    if window_mean:
+        raw = raw / float(ws * G)
+    pooled = avg_pool_same(raw, pool) if pool_kind == 1 else max_pool_same(raw, pool)
+    return {"score": pooled, "raw": raw, "window_mass": wmass}
 
 
 # --------------------------------------------------------------------------- per-head top-k (Eq. 3)
@@ -144,23 +174,35 @@ def global_topk_counts(history: Sequence[np.ndarray], k: int) -> np.ndarray:
     return np.bincount(layer_of, minlength=len(history)).astype(np.int64)
 
 
-def budget_from_counts(cnt: Sequence[int], Bl: int, N: int, L: int) -> Dict[str, List[int]]:
+def budget_from_counts(cnt: Sequence[int], Bl: int, N: int, L: int, *, prorata: bool = False,
+                       minmax: bool = False) -> Dict[str, List[int]]:
     """Eq. 5 and Eq. 6 with Update_Buffer_Length's integer truncations.
 
     ``Z_i = floor(Bl * cnt_i / max(cnt))`` (any positive normalisation of the counts cancels),
     ``Z'_i = floor(Z_i * (N * L) / sum(Z))`` with ``B = N * L`` the global budget.
+
+    Variant readings: ``prorata`` uses the budget of the layers seen so far, ``B = N * len(cnt)``, at an
+    intermediate update; ``minmax`` reads "Norm ... range in (0,1)" as min-max normalisation,
+    ``t_i = (cnt_i - min) / (max - min)`` (all ``t_i = 1`` when every layer has the same count), so that
+    ``Z_i = floor(Bl * (cnt_i - min) / (max - min))``.
     """
     c = [int(x) for x in cnt]
     cmax = max(c)
     if cmax <= 0:
         raise ValueError("no hits in any layer")
-    Z = [(int(Bl) * t) // cmax for t in c]
+    if minmax:
+        cmin = min(c)
+        Z = [int(Bl)] * len(c) if cmax == cmin else [(int(Bl) * (t - cmin)) // (cmax - cmin) for t in c]
+    else:
+        Z = [(int(Bl) * t) // cmax for t in c]
     total = sum(Z)
-    Zp = [(z * int(N) * int(L)) // total for z in Z]
+    B = int(N) * (len(c) if prorata else int(L))
+    Zp = [(z * B) // total for z in Z]
     return {"Z": Z, "Zp": Zp}
 
 
-def rebudget(history: Sequence[np.ndarray], counts: Sequence[int], N: int, Bl: int, L: int) -> Dict[str, List[int]]:
+def rebudget(history: Sequence[np.ndarray], counts: Sequence[int], N: int, Bl: int, L: int, *,
+             prorata: bool = False, minmax: bool = False) -> Dict[str, List[int]]:
     """Update_Buffer_Length after ``l = len(history)`` layers for one sample.
 
     ``k = N * H * l`` entries are selected globally (all of them if fewer exist).  The new count of
@@ -170,7 +212,7 @@ def rebudget(history: Sequence[np.ndarray], counts: Sequence[int], N: int, Bl: i
     H, P = np.asarray(history[0]).shape
     k = min(int(N) * H * l, l * H * P)
     cnt = global_topk_counts(history, k)
-    zz = budget_from_counts(cnt, Bl, N, L)
+    zz = budget_from_counts(cnt, Bl, N, L, prorata=prorata, minmax=minmax)
     new_counts = [int(x) for x in counts]
     for i in range(l):
         new_counts[i] = min(new_counts[i], zz["Zp"][i])
@@ -190,7 +232,8 @@ def shrink_rows(buf: np.ndarray, idx: np.ndarray, rank: np.ndarray, valid: int, 
     return rows, idx[keep], rank[keep]
 
 
-def run_prefill_pass(layer_fn, L: int, *, ws: int, pool: int, N: int, Bl: int, m: int) -> Dict[str, object]:
+def run_prefill_pass(layer_fn, L: int, *, ws: int, pool: int, N: int, Bl: int, m: int, pool_kind: int = 0,
+                     window_mean: bool = False, prorata: bool = False, minmax: bool = False) -> Dict[str, object]:
     """Algorithm 1's loop over the layers, for all samples.
 
     ``layer_fn(l)`` returns one layer's inputs as a dict: ``q`` [Bt,Hq,ws,D] and ``k`` [Bt,Hkv,S,D]
@@ -213,7 +256,7 @@ def run_prefill_pass(layer_fn, L: int, *, ws: int, pool: int, N: int, Bl: int, m
         trail = []
         Bt, Hkv = counts.shape[0], len(idx[0][0])
         for b in range(Bt):
-            res = rebudget([scores[i][b] for i in range(l_done)], counts[b], N, Bl, L)
+            res = rebudget([scores[i][b] for i in range(l_done)], counts[b], N, Bl, L, prorata=prorata, minmax=minmax)
             for i in range(l_done):
                 new = res["counts"][i]
                 valid = int(counts[b, i])
@@ -232,7 +275,7 @@ def run_prefill_pass(layer_fn, L: int, *, ws: int, pool: int, N: int, Bl: int, m
         P = S - ws
         if counts is None:
             counts = np.zeros((Bt, L), dtype=np.int64)
-        sc = window_scores(inp["q"], inp["k"], ws, pool)["score"]
+        sc = window_scores(inp["q"], inp["k"], ws, pool, pool_kind=pool_kind, window_mean=window_mean)["score"]
         scores.append(sc)
         for lst in (idx, rank, kb, vb, first_idx, first_rank):
             lst.append([[None] * Hkv for _ in range(Bt)])
