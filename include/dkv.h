@@ -45,6 +45,16 @@ extern "C" {
 #define DKV_MAX_LAYER_BUDGET  16384  /* Bl  */
 #define DKV_MAX_WINDOW_ROWS   256    /* ws * G */
 
+/* Alternative readings of passages where the paper is silent or inconsistent (dkv_config.flags).
+ * With all bits clear the library computes the default readings.                                  */
+#define DKV_F_WINDOW_MEAN  0x1u  /* Algorithm 1's scoring line takes the MEAN over the window rows (and the
+                                    query heads of a group) where Eq. 2 is read as a sum: scores / (ws*G)  */
+#define DKV_F_PRORATA      0x2u  /* Eq. 6 at an update after l < L layers uses the budget of those layers,
+                                    B = (wt-ws)*l, instead of (wt-ws)*L                                    */
+#define DKV_F_NORM_MINMAX  0x4u  /* Update_Buffer_Length's "Norm ... range in (0,1)" is min-max scaling:
+                                    t_i = (cnt_i - min)/(max - min), all 1 if every layer counts the same  */
+#define DKV_F_ALL          0x7u
+
 typedef struct dkv_ctx dkv_ctx;     /* opaque; owns score history, kept indices, ranks, counts, workspace */
 
 /* Problem statement of Algorithm 1 (its inputs r_max, m, wt, ws, S, d_k) plus the model shape. */
@@ -57,11 +67,11 @@ typedef struct {
   int32_t seq_len;          /* S   : includes the window; S > ws                                  */
   int32_t window;           /* ws  : ws * G <= DKV_MAX_WINDOW_ROWS                                */
   int32_t pool_kernel;      /* odd width of the 1-D pooling of Eq. 2, 1..255                      */
-  int32_t pool_kind;        /* 0 = max-pool (only kind built)                                     */
+  int32_t pool_kind;        /* 0 = max-pool (default), 1 = average over the neighbours that exist */
   int32_t avg_budget;       /* N = wt - ws : retained prefix tokens per head per layer on average */
   int32_t layer_max;        /* Bl = floor(N * r_max), N <= Bl <= DKV_MAX_LAYER_BUDGET             */
   int32_t update_interval;  /* m >= 1                                                             */
-  uint32_t flags;           /* must be 0                                                          */
+  uint32_t flags;           /* DKV_F_* bits, 0 = the default readings                             */
 } dkv_config;
 
 /* Create a context for `cfg` on the current device (host call; allocates device memory:

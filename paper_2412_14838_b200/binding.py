@@ -123,13 +123,19 @@ def _check(code: int, what: str) -> None:
         raise DkvError(code, what)
 
 
+# dkv_config.flags: alternative readings of the paper (see include/dkv.h)
+DKV_F_WINDOW_MEAN = 0x1
+DKV_F_PRORATA = 0x2
+DKV_F_NORM_MINMAX = 0x4
+
+
 def make_config(L, Hq, Hkv, D, Bt, S, ws, pool, N, Bl, m, pool_kind=0, flags=0) -> DkvConfig:
     return DkvConfig(L, Hq, Hkv, D, Bt, S, ws, pool, pool_kind, N, Bl, m, flags)
 
 
-def config_of(w) -> DkvConfig:
+def config_of(w, pool_kind: int = 0, flags: int = 0) -> DkvConfig:
     """DkvConfig of a ``synth.Workload``-like object (fields L,Hq,Hkv,D,Bt,S,ws,pool,N,Bl,m)."""
-    return make_config(w.L, w.Hq, w.Hkv, w.D, w.Bt, w.S, w.ws, w.pool, w.N, w.Bl, w.m)
+    return make_config(w.L, w.Hq, w.Hkv, w.D, w.Bt, w.S, w.ws, w.pool, w.N, w.Bl, w.m, pool_kind, flags)
 
 
 # ---- the entry points, same names as the C ABI ----------------------------------------------------

@@ -119,8 +119,8 @@ int validate(const dkv_config* c) {
   if (c->pool_kernel < 1 || c->pool_kernel % 2 == 0) return DKV_ERR_INVALID_ARG;
   if (c->pool_kernel > 255) return DKV_ERR_UNSUPPORTED;
   if (c->avg_budget < 1 || c->layer_max < c->avg_budget || c->update_interval < 1) return DKV_ERR_INVALID_ARG;
-  if (c->flags != 0) return DKV_ERR_INVALID_ARG;
-  if (c->pool_kind != 0) return DKV_ERR_UNSUPPORTED;
+  if (c->flags & ~DKV_F_ALL) return DKV_ERR_INVALID_ARG;
+  if (c->pool_kind != 0 && c->pool_kind != 1) return DKV_ERR_UNSUPPORTED;
   if (c->n_layers > DKV_MAX_LAYERS || c->layer_max > DKV_MAX_LAYER_BUDGET) return DKV_ERR_UNSUPPORTED;
   if (c->head_dim != 64 && c->head_dim != 128) return DKV_ERR_UNSUPPORTED;
   if ((long long)c->window * (c->n_q_heads / c->n_kv_heads) > DKV_MAX_WINDOW_ROWS) return DKV_ERR_UNSUPPORTED;
@@ -188,6 +188,8 @@ bool make_job(dkv_ctx* c, int mode, int layer, const void* q, const void* k, flo
   p->status = c->d_status;
   p->stats_grid = c->tc_grid;
   p->mode = mode;
+  p->out_scale = (c->cfg.flags & DKV_F_WINDOW_MEAN) ? 1.0f / (float)s.M : 1.0f;
+  p->pool_avg = c->cfg.pool_kind == 1;
   p->idesc = mode == tc::kStats ? make_idesc(128, 128) : make_idesc(128, p->nq16);
   return true;
 }
@@ -270,7 +272,7 @@ int do_rebudget(dkv_ctx* c, int l, int* counts_out, cudaStream_t st) {
   const size_t bl = (size_t)s.Bt * s.L;
   rb_budget_kernel<<<s.Bt, 1024, 0, st>>>(c->d_rb_state, c->d_rb_hist1, c->d_rb_above, c->d_rb_above2, c->d_rb_hist2,
                                          c->d_count, c->d_dbg, c->d_dbg + bl, c->d_dbg + 2 * bl, counts_out, s.Bt, s.L, l,
-                                         s.Bl, s.N);
+                                         s.Bl, s.N, (c->cfg.flags & DKV_F_PRORATA) != 0, (c->cfg.flags & DKV_F_NORM_MINMAX) != 0);
   DKV_LAUNCHED(c);
   for (int i = 0; i < l; ++i) if (!c->gathered[i]) c->stale[i] = 1;
   return DKV_OK;
@@ -759,6 +761,8 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   p.tph = tph; p.nq16 = (M + 15) / 16 * 16; p.nmblk = (M + 127) / 128;
   p.slots = slots; p.m_stride = 256;
   p.scale2 = kLog2e / sqrtf((float)D);
+  p.out_scale = (cfg->flags & DKV_F_WINDOW_MEAN) ? 1.0f / (float)M : 1.0f;
+  p.pool_avg = cfg->pool_kind == 1;
   p.stats = reinterpret_cast<float2*>(su.ptr + 256);
   p.scores = scores_out; p.copy_out = nullptr;
   p.status = reinterpret_cast<int*>(su.ptr);

@@ -141,7 +141,7 @@ rb_budget_kernel(const RbState* __restrict__ state, const unsigned int* __restri
                  const unsigned int* __restrict__ above, const unsigned int* __restrict__ above2,
                  const unsigned int* __restrict__ hist2, int* __restrict__ count, int* __restrict__ dbg_cnt,
                  int* __restrict__ dbg_z, int* __restrict__ dbg_zp, int* __restrict__ counts_out,
-                 int Bt, int L, int l, int Bl, int N) {
+                 int Bt, int L, int l, int Bl, int N, int prorata, int minmax) {
   __shared__ unsigned int sh[kBins];
   __shared__ int sm_scan[33];
   __shared__ int found[2];
@@ -179,7 +179,7 @@ rb_budget_kernel(const RbState* __restrict__ state, const unsigned int* __restri
   // Eq. 5-6 with one thread per layer (warp 0; layers lane, lane + 32, ...): the ties go to the lowest layers
   // first, i.e. layer i takes min(eq_i, ties - sum of eq below i).
   if (warp == 0) {
-    long long carry = 0, cmax = 0;
+    long long carry = 0, cmax = 0, cmin = 0x7FFFFFFFFFFFFFFFll;
     for (int i0 = 0; i0 < l; i0 += 32) {
       const int i = i0 + lane;
       const long long eq = i < l ? s_eq[i] : 0;
@@ -193,22 +193,27 @@ rb_budget_kernel(const RbState* __restrict__ state, const unsigned int* __restri
         s_gt[i] += take;                      // = cnt_i
         dbg_cnt[b * L + i] = (int)s_gt[i];
         cmax = s_gt[i] > cmax ? s_gt[i] : cmax;
+        cmin = s_gt[i] < cmin ? s_gt[i] : cmin;
       }
       carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) { const long long y = __shfl_xor_sync(0xFFFFFFFFu, cmax, o); cmax = y > cmax ? y : cmax; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { const long long y = __shfl_xor_sync(0xFFFFFFFFu, cmin, o); cmin = y < cmin ? y : cmin; }
     if (cmax <= 0) cmax = 1;
     long long sumz = 0;
     for (int i = lane; i < l; i += 32) {
-      s_eq[i] = ((long long)Bl * s_gt[i]) / cmax;             // Z_i
+      // Z_i: counts scaled by their maximum, or (variant) min-max scaled; all layers equal under min-max -> Bl each
+      if (minmax) s_eq[i] = cmax == cmin ? (long long)Bl : ((long long)Bl * (s_gt[i] - cmin)) / (cmax - cmin);
+      else s_eq[i] = ((long long)Bl * s_gt[i]) / cmax;
       dbg_z[b * L + i] = (int)s_eq[i];
       sumz += s_eq[i];
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sumz += __shfl_xor_sync(0xFFFFFFFFu, sumz, o);
     if (sumz <= 0) sumz = 1;
-    const long long B = (long long)N * L;
+    const long long B = (long long)N * (prorata ? l : L);      // Eq. 6's budget (variant: of the layers seen so far)
     for (int i = lane; i < l; i += 32) {
       const long long zp = (s_eq[i] * B) / sumz;              // Z'_i
       const int zpi = zp > 0x7FFFFFFF ? 0x7FFFFFFF : (int)zp;

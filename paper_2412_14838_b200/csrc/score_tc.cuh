@@ -56,6 +56,8 @@ struct Params {
   int* status;             // device status words; [0] = first error
   int stats_grid;          // CTAs of the launch that ran sweep 1 for this layer
   int mode;                // kNone: nothing to do
+  float out_scale;         // sweep 2: factor on the raw scores before pooling (1, or 1/(ws*G) for the window mean)
+  int pool_avg;            // sweep 2: 0 = max-pool, 1 = average over the neighbours that exist
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -495,15 +497,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
           asm volatile("bar.sync 1, 512;" ::: "memory");
           // add up the two column halves in a fixed order; raw_s[x] then belongs to key key0 + x
           for (int x = sid; x < sg.ntiles * kTileKeys; x += kSoftmaxThreads)
-            raw_s[x] += raw_s[kMaxSegTiles * kTileKeys + x];
+            raw_s[x] = (raw_s[x] + raw_s[kMaxSegTiles * kTileKeys + x]) * p.out_scale;
           asm volatile("bar.sync 1, 512;" ::: "memory");
           // Eq. 2's pooling over this segment
           for (int o = sg.out0 + sid; o < sg.out1; o += kSoftmaxThreads) {
             const int x = o - sg.key0;
             float v = raw_s[x];
-            for (int d = 1; d <= p.half; ++d) {
-              if (o - d >= 0) v = fmaxf(v, raw_s[x - d]);
-              if (o + d < p.P) v = fmaxf(v, raw_s[x + d]);
+            if (p.pool_avg) {
+              int cnt = 1;
+              for (int d = 1; d <= p.half; ++d) {
+                if (o - d >= 0) { v += raw_s[x - d]; ++cnt; }
+                if (o + d < p.P) { v += raw_s[x + d]; ++cnt; }
+              }
+              v = v / (float)cnt;
+            } else {
+              for (int d = 1; d <= p.half; ++d) {
+                if (o - d >= 0) v = fmaxf(v, raw_s[x - d]);
+                if (o + d < p.P) v = fmaxf(v, raw_s[x + d]);
+              }
             }
             const size_t at = (size_t)sg.bh * p.P + o;
             p.scores[at] = v;

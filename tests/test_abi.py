@@ -48,8 +48,8 @@ def test_version_and_strerror(lib):
     (dict(L=500), binding.DKV_ERR_UNSUPPORTED),
     (dict(Bl=100000), binding.DKV_ERR_UNSUPPORTED),
     (dict(ws=128, S=4096), binding.DKV_ERR_UNSUPPORTED),  # ws*G = 512 window rows
-    (dict(pool_kind=1), binding.DKV_ERR_UNSUPPORTED),
-    (dict(flags=1), binding.DKV_ERR_INVALID_ARG),
+    (dict(pool_kind=2), binding.DKV_ERR_UNSUPPORTED),     # 0 = max, 1 = average
+    (dict(flags=0x100), binding.DKV_ERR_INVALID_ARG),     # not one of the DKV_F_* bits
 ])
 def test_bad_configs_are_rejected_on_the_host(lib, kw, code):
     base = dict(L=4, Hq=8, Hkv=2, D=64, Bt=1, S=1024, ws=16, pool=5, N=64, Bl=128, m=2)

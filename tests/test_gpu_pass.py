@@ -33,8 +33,9 @@ def dev(bits):
 class GpuPass:
     """Inputs on the device, one full pass, results back on the host."""
 
-    def __init__(self, w, keep_inputs=True):
+    def __init__(self, w, keep_inputs=True, pool_kind=0, flags=0):
         self.w = w
+        self.pool_kind, self.flags = pool_kind, flags
         self.q, self.k, self.v = [], [], []
         self.host = []
         for l in range(w.L):
@@ -44,7 +45,7 @@ class GpuPass:
         shape = (w.Bt, w.Hkv, w.Blc + w.ws, w.D)
         self.kb = [torch.zeros(shape, dtype=torch.int16, device="cuda") for _ in range(w.L)]
         self.vb = [torch.zeros(shape, dtype=torch.int16, device="cuda") for _ in range(w.L)]
-        self.h = B.dkv_create(B.config_of(w))
+        self.h = B.dkv_create(B.config_of(w, pool_kind, flags))
 
     def run(self):
         B.dkv_run_prefill_pass(self.h, self.q, self.k, self.v, self.kb, self.vb)
@@ -115,7 +116,9 @@ def compare_full(g: GpuPass, verbose_name=""):
         return {"q": synth.bf16_bits_to_f64(t["q"]), "k": synth.bf16_bits_to_f64(t["k"]),
                 "k_rows": t["k"], "v_rows": t["v"]}
 
-    ref = O.run_prefill_pass(layer_fn, w.L, ws=w.ws, pool=w.pool, N=w.N, Bl=w.Bl, m=w.m)
+    ref = O.run_prefill_pass(layer_fn, w.L, ws=w.ws, pool=w.pool, N=w.N, Bl=w.Bl, m=w.m, pool_kind=g.pool_kind,
+                             window_mean=bool(g.flags & B.DKV_F_WINDOW_MEAN), prorata=bool(g.flags & B.DKV_F_PRORATA),
+                             minmax=bool(g.flags & B.DKV_F_NORM_MINMAX))
     worst, near = 0.0, 0
     for l in range(w.L):
         worst = max(worst, U.assert_scores_close(g.scores(l), ref["score"][l], f"{w.name} layer {l}"))
