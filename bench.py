@@ -39,10 +39,10 @@ NOMINAL_HBM_GBS = 8000.0
 # every replay starts from flushed caches.  Both hold for the kernel source they were measured on and for that
 # per-layer shape only: any other source hash or shape reports null.
 NCU_TRAFFIC = {
-    "kernel_sha256": "8d25d862828a65fe10202e1e0f01f86703778af2175c0320a8c36b199c2f5c04",
+    "kernel_sha256": "f3ebfc768f27dfa9d6af7f839f8753d7e2be972a44665d7b5208e04b690248e7",
     "shape": (8, 128, 1, 32768, 32),          # Hkv, D, Bt, S, ws
-    "live_bytes_per_launch": 76_730_000 + 10_460_000,
-    "cold_bytes_per_launch": 134_960_000 + 4_280_000,
+    "live_bytes_per_launch": 76_640_000 + 10_230_000,
+    "cold_bytes_per_launch": 134_960_000 + 4_050_000,
 }
 
 

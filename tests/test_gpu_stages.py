@@ -59,6 +59,8 @@ SHAPES = [
     synth.Workload("rag4", 14, L=1, Hq=4, Hkv=2, D=64, Bt=1, S=20, ws=16, pool=9, N=2, Bl=4, m=1, recipe="iid"),
     # 16 window rows = a single 16-column chunk in sweep 2 (half of the softmax warps have nothing to read),
     # one head long enough that every CTA reuses its accumulator stages
+    # G = 7 (28 query / 4 KV heads scaled down): 224 window rows, not a power of two, two row blocks in sweep 1
+    synth.Workload("rag6", 17, L=1, Hq=14, Hkv=2, D=128, Bt=1, S=2500, ws=32, pool=7, N=8, Bl=16, m=1, recipe="sink"),
     synth.Workload("rag5", 16, L=1, Hq=2, Hkv=1, D=64, Bt=1, S=90001, ws=8, pool=3, N=8, Bl=16, m=1, recipe="iid"),
 ]
 
