@@ -161,7 +161,11 @@ int dkv_compact_all(dkv_ctx* ctx, int32_t upto_layer, void* const* kb, void* con
 
 /* Algorithm 1's loop over all L layers: score, select, gather each layer; after every m-th layer (and
  * after the last one if L % m != 0) rebudget and shrink all preceding layers.  Resets the context first.
- * q_win, k, v, kb, vb : HOST arrays of L device pointers (layouts as above). */
+ * q_win, k, v, kb, vb : HOST arrays of L device pointers (layouts as above).
+ * The first call with a given set of pointers records the whole pass as a CUDA graph (on an internal stream
+ * that forks from `stream` and rejoins it); later calls with the same pointers replay it, whatever the
+ * buffers then contain.  The plain sequence of launches is used instead while dkv_profile is on, when
+ * `stream` is itself being captured, or if the capture fails. */
 int dkv_run_prefill_pass(dkv_ctx* ctx, const void* const* q_win, const void* const* k, const void* const* v,
                          void* const* kb, void* const* vb, void* stream);
 

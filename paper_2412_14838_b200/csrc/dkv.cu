@@ -52,6 +52,13 @@ struct dkv_ctx {
   // host state
   uint8_t scored[DKV_MAX_LAYERS], selected[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
   long long launches;
+  // dkv_run_prefill_pass as a CUDA graph: captured on the first call with a set of pointers, replayed afterwards
+  bool use_graph;
+  cudaStream_t gstream;        // the graph is captured and replayed here, forked from / joined to the caller's stream
+  cudaEvent_t ev_gfork, ev_gjoin;
+  cudaGraphExec_t pass_exec;
+  std::vector<const void*>* pass_key;
+  long long pass_launches;
   int last_cuda;
   // optional per-step timing with CUDA events (dkv_profile)
   bool prof_on;
@@ -381,6 +388,11 @@ void free_all(dkv_ctx* c) {
   cudaFree(c->d_cand); cudaFree(c->d_cand_n); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
   for (int i = 0; i < 2; ++i) if (c->side[i]) cudaStreamDestroy(c->side[i]);
   if (c->hi) cudaStreamDestroy(c->hi);
+  if (c->pass_exec) cudaGraphExecDestroy(c->pass_exec);
+  delete c->pass_key;
+  if (c->gstream) cudaStreamDestroy(c->gstream);
+  if (c->ev_gfork) cudaEventDestroy(c->ev_gfork);
+  if (c->ev_gjoin) cudaEventDestroy(c->ev_gjoin);
   if (c->upd) cudaStreamDestroy(c->upd);
   for (int i = 0; i < 3; ++i) if (c->ev_join[i]) cudaEventDestroy(c->ev_join[i]);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
@@ -502,6 +514,12 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * 3 * heads * c->tc_slots * 256));
   TRY(cudaFuncSetAttribute(tc::score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   for (int i = 0; i < 2; ++i) TRY(cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking));
+  TRY(cudaStreamCreateWithFlags(&c->gstream, cudaStreamNonBlocking));
+  TRY(cudaEventCreateWithFlags(&c->ev_gfork, cudaEventDisableTiming));
+  TRY(cudaEventCreateWithFlags(&c->ev_gjoin, cudaEventDisableTiming));
+  c->pass_key = new (std::nothrow) std::vector<const void*>();
+  if (!c->pass_key) { free_all(c); delete c; return DKV_ERR_NOMEM; }
+  c->use_graph = getenv("DKV_NO_GRAPH") == nullptr;
   TRY(cudaStreamCreateWithFlags(&c->upd, cudaStreamNonBlocking));
   {
     int least = 0, greatest = 0;
@@ -624,7 +642,49 @@ int dkv_run_prefill_pass(dkv_ctx* c, const void* const* q_win, const void* const
     if (!aligned16(q_win[l]) || !aligned16(k[l]) || !aligned16(v[l]) || !aligned16(kb[l]) || !aligned16(vb[l]))
       return DKV_ERR_INVALID_ARG;
   }
-  return do_pass(c, q_win, k, v, kb, vb, as_stream(stream));
+  cudaStream_t st = as_stream(stream);
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
+  // per-step profiling needs its events between the launches; a caller that is capturing gets the plain calls
+  if (!c->use_graph || c->prof_on || cap != cudaStreamCaptureStatusNone) return do_pass(c, q_win, k, v, kb, vb, st);
+
+  std::vector<const void*> key;
+  key.reserve(5 * (size_t)c->s.L);
+  for (int l = 0; l < c->s.L; ++l) { key.push_back(q_win[l]); key.push_back(k[l]); key.push_back(v[l]); key.push_back(kb[l]); key.push_back(vb[l]); }
+  if (!c->pass_exec || *c->pass_key != key) {
+    // first call with these buffers: record the whole pass (all streams of do_pass fork from and rejoin gstream)
+    if (c->pass_exec) { cudaGraphExecDestroy(c->pass_exec); c->pass_exec = nullptr; }
+    const long long before = c->launches;
+    cudaGraph_t graph = nullptr;
+    DKV_CUDA(c, cudaStreamBeginCapture(c->gstream, cudaStreamCaptureModeThreadLocal));
+    const int rc = do_pass(c, q_win, k, v, kb, vb, c->gstream);
+    const cudaError_t e = cudaStreamEndCapture(c->gstream, &graph);
+    if (rc != DKV_OK || e != cudaSuccess || !graph) {
+      if (graph) cudaGraphDestroy(graph);
+      cudaGetLastError();
+      c->launches = before;
+      c->use_graph = false;                         // not capturable here: run the plain calls from now on
+      return do_pass(c, q_win, k, v, kb, vb, st);
+    }
+    c->pass_launches = c->launches - before;
+    c->launches = before;
+    const cudaError_t ei = cudaGraphInstantiate(&c->pass_exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ei != cudaSuccess) {
+      cudaGetLastError();
+      c->pass_exec = nullptr; c->use_graph = false;
+      return do_pass(c, q_win, k, v, kb, vb, st);
+    }
+    *c->pass_key = key;
+  }
+  DKV_CUDA(c, cudaEventRecord(c->ev_gfork, st));
+  DKV_CUDA(c, cudaStreamWaitEvent(c->gstream, c->ev_gfork, 0));
+  DKV_CUDA(c, cudaGraphLaunch(c->pass_exec, c->gstream));
+  DKV_CUDA(c, cudaEventRecord(c->ev_gjoin, c->gstream));
+  DKV_CUDA(c, cudaStreamWaitEvent(st, c->ev_gjoin, 0));
+  c->launches += c->pass_launches;
+  for (int l = 0; l < c->s.L; ++l) { c->scored[l] = c->selected[l] = c->gathered[l] = 1; c->stale[l] = 0; }
+  return DKV_OK;
 }
 
 int dkv_run_prefill_pass_host(dkv_ctx* c, const void* const* q_win, const void* const* k, const void* const* v,

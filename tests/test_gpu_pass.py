@@ -239,3 +239,30 @@ def test_host_buffer_pass_matches_device_pass():
                 assert torch.equal(ovb[l][:, :, :n], g.vb[l].cpu()[:, :, :n])
     finally:
         g.close()
+
+
+def test_pass_replayed_and_recaptured_gives_the_same_result():
+    """The pass is recorded as a CUDA graph on its first call and replayed afterwards; a call with other
+    buffers records again.  All three must produce the same counts, indices and bytes."""
+    w = synth.WORKLOADS["tiny"]
+    g = GpuPass(w).run()
+    try:
+        counts0 = g.counts.copy()
+        idx0 = [g.kept(l)[1].copy() for l in range(w.L)]
+        kb0 = [x.clone() for x in g.kb]
+        for x in g.kb:
+            x.zero_()
+        g.run()                                           # replay
+        assert (g.counts == counts0).all()
+        for l in range(w.L):
+            assert (g.kept(l)[1] == idx0[l]).all()
+            n = int(counts0[0, l]) + w.ws
+            assert torch.equal(g.kb[l][:, :, :n], kb0[l][:, :, :n])
+        g.kb = [torch.zeros_like(x) for x in g.kb]        # other output buffers: recorded again
+        g.run()
+        assert (g.counts == counts0).all()
+        for l in range(w.L):
+            n = int(counts0[0, l]) + w.ws
+            assert torch.equal(g.kb[l][:, :, :n], kb0[l][:, :, :n])
+    finally:
+        g.close()
