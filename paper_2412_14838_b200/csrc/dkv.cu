@@ -48,7 +48,7 @@ struct dkv_ctx {
                         // waiting scoring CTA before the side streams' many short CTAs
   cudaStream_t upd;     // budget updates (rebudget + shrink) of dkv_run_prefill_pass, off the select streams
   cudaStream_t side[2]; // side streams of dkv_run_prefill_pass (select / gather / rebudget / shrink), layers alternate
-  cudaEvent_t ev_fork, ev_join[3], ev_update, ev_scored[DKV_MAX_LAYERS], ev_selected[DKV_MAX_LAYERS];
+  cudaEvent_t ev_fork, ev_join[3], ev_update, ev_scored[DKV_MAX_LAYERS], ev_picked[DKV_MAX_LAYERS], ev_selected[DKV_MAX_LAYERS];
   // host state
   uint8_t scored[DKV_MAX_LAYERS], selected[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
   long long launches;
@@ -357,16 +357,19 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
     DKV_CUDA(c, cudaEventRecord(c->ev_scored[el], st));
     DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_scored[el], 0));
     if ((rc = do_select(c, el, nullptr, nullptr, sd))) return rc;
+    DKV_CUDA(c, cudaEventRecord(c->ev_picked[el], sd));
     if ((rc = do_gather(c, el, k[el], v[el], kb[el], vb[el], sd))) return rc;
     DKV_CUDA(c, cudaEventRecord(c->ev_selected[el], sd));
     const bool update = ((el + 1) % s.m == 0) || (el + 1 == s.L && s.L % s.m != 0);
     if (update) {
-      // needs every earlier layer selected and gathered (both select streams, each in layer order); the
-      // previous update precedes it on the same stream.  Later layers' select and gather do not wait for it:
-      // an update changes the counts and buffers of the layers before it only.
+      // The rebudget needs every earlier layer selected (both select streams, each in layer order), the shrink
+      // also gathered; the previous update precedes it on the same stream.  Later layers' select and gather
+      // do not wait for it: an update changes the counts and buffers of the layers before it only.
+      DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_picked[el], 0));
+      if (el >= 1) DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_picked[el - 1], 0));
+      if ((rc = do_rebudget(c, el + 1, nullptr, c->upd))) return rc;
       DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_selected[el], 0));
       if (el >= 1) DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_selected[el - 1], 0));
-      if ((rc = do_rebudget(c, el + 1, nullptr, c->upd))) return rc;
       if ((rc = do_shrink(c, 0, el + 1, kb, vb, c->upd))) return rc;
     }
   }
@@ -400,6 +403,7 @@ void free_all(dkv_ctx* c) {
   for (int l = 0; l < DKV_MAX_LAYERS; ++l) {
     if (c->ev_scored[l]) cudaEventDestroy(c->ev_scored[l]);
     if (c->ev_selected[l]) cudaEventDestroy(c->ev_selected[l]);
+    if (c->ev_picked[l]) cudaEventDestroy(c->ev_picked[l]);
   }
   if (c->prof_recs) {
     for (ProfRec& r : *c->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -532,6 +536,7 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   for (int l = 0; l < s.L; ++l) {
     TRY(cudaEventCreateWithFlags(&c->ev_scored[l], cudaEventDisableTiming));
     TRY(cudaEventCreateWithFlags(&c->ev_selected[l], cudaEventDisableTiming));
+    TRY(cudaEventCreateWithFlags(&c->ev_picked[l], cudaEventDisableTiming));
   }
   TRY(cudaMalloc(&c->d_status, sizeof(int) * 8));
   TRY(cudaMemset(c->d_status, 0, sizeof(int) * 8));

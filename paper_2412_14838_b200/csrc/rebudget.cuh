@@ -70,39 +70,50 @@ rb_locate_kernel(const unsigned int* __restrict__ layer_hist, RbState* __restric
 // grid (slices, l, Bt): one pass over the scores of layers [0, l).  Scores whose first digit is b* go to the
 // sample's candidate list (value, layer) and into the second-digit histogram.  The list has room for every
 // score (cand[b] holds l*Hkv*P pairs at most); its order is arbitrary, only counts are taken from it.
+// A block reads its slice once, in chunks of kRbChunk scores: matches are parked in shared memory, then the
+// block reserves a range of the list with one atomic and copies them out.
+constexpr int kRbChunk = 4096;
 __global__ void __launch_bounds__(kRbThreads)
 rb_refine1_kernel(const float* __restrict__ scores, const RbState* __restrict__ state, unsigned int* __restrict__ hist1,
                   uint2* __restrict__ cand, unsigned int* __restrict__ cand_n, int Bt, size_t per_layer /* Hkv*P */,
                   size_t cand_stride) {
   __shared__ unsigned int sh[kBins];
+  __shared__ uint32_t parked[kRbChunk];
   __shared__ unsigned int s_cnt, s_base;
   const int b = blockIdx.z, i = blockIdx.y;
   const uint32_t d = (uint32_t)state[b].bstar;
   const uint32_t* v = reinterpret_cast<const uint32_t*>(scores) + ((size_t)i * Bt + b) * per_layer;
   for (int j = threadIdx.x; j < kBins; j += kRbThreads) sh[j] = 0;
-  if (threadIdx.x == 0) s_cnt = 0;
-  __syncthreads();
-  // two sweeps over this block's slice: count, reserve a range of the list, then fill it
   const size_t per_block = (per_layer + gridDim.x - 1) / gridDim.x;
   const size_t e0 = (size_t)blockIdx.x * per_block, e1 = e0 + per_block < per_layer ? e0 + per_block : per_layer;
-  unsigned int mine = 0;
-  for (size_t e = e0 + threadIdx.x; e < e1; e += kRbThreads) mine += ((v[e] >> 21) == d);
-  if (mine) atomicAdd(&s_cnt, mine);
-  __syncthreads();
-  const unsigned int block_total = s_cnt;
-  __syncthreads();
-  if (block_total == 0) return;
-  if (threadIdx.x == 0) { s_base = atomicAdd(&cand_n[b], block_total); s_cnt = 0; }
-  __syncthreads();
   uint2* list = cand + (size_t)b * cand_stride;
-  for (size_t e = e0 + threadIdx.x; e < e1; e += kRbThreads) {
-    const uint32_t u = v[e];
-    if ((u >> 21) == d) {
-      list[s_base + atomicAdd(&s_cnt, 1u)] = make_uint2(u, (unsigned int)i);
-      atomicAdd(&sh[(u >> 10) & 2047u], 1u);
+  for (size_t c0 = e0; c0 < e1; c0 += kRbChunk) {
+    if (threadIdx.x == 0) s_cnt = 0;
+    __syncthreads();
+    const size_t c1 = c0 + kRbChunk < e1 ? c0 + kRbChunk : e1;
+    uint32_t u[kRbChunk / kRbThreads];
+#pragma unroll
+    for (int j = 0; j < kRbChunk / kRbThreads; ++j) {          // all loads of the chunk in flight together
+      const size_t e = c0 + threadIdx.x + (size_t)j * kRbThreads;
+      u[j] = e < c1 ? v[e] : 0xFFFFFFFFu;                      // (a NaN pattern: its first digit 2047 never is b*)
     }
+#pragma unroll
+    for (int j = 0; j < kRbChunk / kRbThreads; ++j) {
+      const size_t e = c0 + threadIdx.x + (size_t)j * kRbThreads;
+      if (e < c1 && (u[j] >> 21) == d) {
+        parked[atomicAdd(&s_cnt, 1u)] = u[j];
+        atomicAdd(&sh[(u[j] >> 10) & 2047u], 1u);
+      }
+    }
+    __syncthreads();
+    const unsigned int n = s_cnt;
+    if (n) {
+      if (threadIdx.x == 0) s_base = atomicAdd(&cand_n[b], n);
+      __syncthreads();
+      for (unsigned int x = threadIdx.x; x < n; x += kRbThreads) list[s_base + x] = make_uint2(parked[x], (unsigned int)i);
+    }
+    __syncthreads();
   }
-  __syncthreads();
   for (int j = threadIdx.x; j < kBins; j += kRbThreads) { const unsigned int c = sh[j]; if (c) atomicAdd(&hist1[(size_t)b * kBins + j], c); }
 }
 
@@ -125,12 +136,18 @@ rb_refine2_kernel(const uint2* __restrict__ cand, const unsigned int* __restrict
   find_digit(sh, kBins, st.cand, st.need1, sm_scan, found, nullptr);
   const uint32_t s2 = (uint32_t)found[0];
   const uint2* list = cand + (size_t)b * cand_stride;
+  // the per-layer counters are few and hot: count in shared memory (sh is free again), one global add per layer
+  __syncthreads();
+  for (int j = threadIdx.x; j < L; j += kRbThreads) sh[j] = 0;
+  __syncthreads();
   for (unsigned int e = blockIdx.x * kRbThreads + threadIdx.x; e < n; e += gridDim.x * kRbThreads) {
     const uint2 c = list[e];
     const uint32_t dd = (c.x >> 10) & 2047u;
-    if (dd > s2) atomicAdd(&above2[b * L + c.y], 1u);
+    if (dd > s2) atomicAdd(&sh[c.y], 1u);
     else if (dd == s2) atomicAdd(&hist2[((size_t)b * L + c.y) * 1024 + (c.x & 1023u)], 1u);
   }
+  __syncthreads();
+  for (int j = threadIdx.x; j < L; j += kRbThreads) { const unsigned int v = sh[j]; if (v) atomicAdd(&above2[b * L + j], v); }
 }
 
 // One CTA of 1024 threads per sample: exact T, per-layer hits, Eq. 5-6.
