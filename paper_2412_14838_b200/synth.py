@@ -89,6 +89,9 @@ WORKLOADS: Dict[str, Workload] = {
                  Bl=256, m=4, recipe="sink"),
         Workload("needle32k", 5, L=32, Hq=32, Hkv=8, D=128, Bt=1, S=32768, ws=32, pool=7, N=64,
                  Bl=512, m=4, recipe="needle"),
+        # a second model shape: 28 layers, 28 query / 4 KV heads (G = 7, 224 window rows: not a power of two)
+        Workload("qwen16k", 6, L=28, Hq=28, Hkv=4, D=128, Bt=1, S=16384, ws=32, pool=7, N=128,
+                 Bl=512, m=4, recipe="sink"),
     ]
 }
 

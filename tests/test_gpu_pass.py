@@ -170,7 +170,7 @@ def test_pass_with_ragged_shape_and_final_partial_block():
         g.close()
 
 
-FULL = ["mistral32k", "llama16k_b4", "needle32k"]
+FULL = ["mistral32k", "llama16k_b4", "needle32k", "qwen16k"]
 
 
 @pytest.mark.parametrize("name", FULL)
