@@ -9,6 +9,7 @@ Each function follows one passage of the paper, in the paper's order and notatio
 prefix tokens, ``N = wt - ws``, ``B^l`` = ``Bl`` per-layer maximum, ``m`` update interval):
 
 * ``window_scores``        Eq. 1-2 and the scoring statement of Algorithm 1.
+* ``window_lse``, ``window_scores_from_lse``  the same scores from Eq. 1's log-denominators (one sweep).
 * ``select_topk``          Eq. 3 and Algorithm 1's per-layer ``topk(B^l)``.
 * ``gather_rows``          Algorithm 1's gather of K/V plus the appended window.
 * ``global_topk_counts``   Eq. 4: top-K over all accumulated layers and the count function Phi.
@@ -31,7 +32,8 @@ lowest index (flat index, layer-major, for the global top-K); ``Norm`` is a posi
 so Eq. 5 is evaluated in exact integers; counts never grow.
 
 Pins (tests/test_oracle_*.py): closed forms for zero keys, probability-mass conservation,
-a hand-worked 3-key softmax, an independent torch softmax / max_pool1d route, permutation
+a hand-worked 3-key softmax, an independent torch softmax / max_pool1d route, torch's logsumexp and the
+ln 6 of the hand-worked case for the log-denominators, permutation
 equivariance, brute-force subset enumeration for the top-k, hand-worked budget cases
 (tests/golden/), full-sort brute force for the global counts, nestedness of shrink, and the
 reduction of the whole pass to a plain top-N when ``r_max = 1`` and ``L = 1``.
@@ -130,6 +132,47 @@ def window_scores(q_win: np.ndarray, k: np.ndarray, ws: int, pool: int, *, pool_
         raw = raw / float(ws * G)
     pooled = avg_pool_same(raw, pool) if pool_kind == 1 else max_pool_same(raw, pool)
     return {"score": pooled, "raw": raw, "window_mass": wmass}
+
+
+def window_lse(q_win: np.ndarray, k: np.ndarray, ws: int) -> np.ndarray:
+    """Natural logarithm of Eq. 1's softmax denominator for every window row: ``lse[b, hq, r] =
+    ln sum_{i <= P + r} exp(q_r . k_i / sqrt(d_k))``, the value a prefill attention kernel returns
+    beside its output.  ``q_win`` [Bt, Hq, ws, D], ``k`` [Bt, Hkv, S, D]; returns [Bt, Hq, ws]."""
+    Bt, Hq, ws_, D = q_win.shape
+    _, Hkv, S, _ = k.shape
+    assert ws_ == ws and Hq % Hkv == 0
+    G, P = Hq // Hkv, S - ws
+    out = np.zeros((Bt, Hq, ws), dtype=np.float64)
+    for b in range(Bt):
+        for hq in range(Hq):
+            logits = (q_win[b, hq] @ k[b, hq // G].T) / np.sqrt(np.float64(D))      # [ws, S]
+            for r in range(ws):
+                row = logits[r, :P + r + 1]
+                top = row.max()
+                out[b, hq, r] = top + np.log(np.exp(row - top).sum())
+    return out
+
+
+def window_scores_from_lse(q_win: np.ndarray, k: np.ndarray, lse: np.ndarray, ws: int, pool: int, *,
+                           pool_kind: int = 0, window_mean: bool = False) -> Dict[str, np.ndarray]:
+    """Eq. 2 with Eq. 1's denominators supplied: ``raw[j] = sum_{g, r} exp(q_{g,r} . k_j / sqrt(d_k) - lse[g, r])``
+    over the prefix keys ``j < P``, then the pooling of ``window_scores``.  With ``lse = window_lse(...)`` this
+    is the same quantity as ``window_scores`` computes by normalising each row."""
+    Bt, Hq, ws_, D = q_win.shape
+    _, Hkv, S, _ = k.shape
+    assert ws_ == ws and Hq % Hkv == 0 and lse.shape == (Bt, Hq, ws)
+    G, P = Hq // Hkv, S - ws
+    raw = np.zeros((Bt, Hkv, P), dtype=np.float64)
+    for b in range(Bt):
+        for h in range(Hkv):
+            for g in range(G):
+                hq = h * G + g
+                logits = (q_win[b, hq] @ k[b, h, :P].T) / np.sqrt(np.float64(D))     # [ws, P]
+                raw[b, h] += np.exp(logits - lse[b, hq][:, None]).sum(axis=0)
+    if window_mean:
+        raw = raw / float(ws * G)
+    pooled = avg_pool_same(raw, pool) if pool_kind == 1 else max_pool_same(raw, pool)
+    return {"score": pooled, "raw": raw}
 
 
 # --------------------------------------------------------------------------- per-head top-k (Eq. 3)
