@@ -122,6 +122,18 @@ int dkv_score(dkv_ctx* ctx, int32_t layer, const void* q_win, const void* k, flo
 #define DKV_STATIC_SCRATCH_BYTES (4u << 20)
 int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, float* scores_out, void* stream);
 
+/* (1') Eq. 2 with Eq. 1's denominators given.  A prefill attention kernel that has just run over the prompt
+ * already holds, for every query row, the logarithm of its softmax denominator (the "log-sum-exp" such
+ * kernels return beside their output).  With those values for the ws window rows the scores of step (1)
+ * need one sweep over the keys instead of two:
+ *       raw[j] = sum over the group's G query heads and the ws window rows r of exp(q . k_j / sqrt(D) - lse[.., r]),
+ * pooled as in step (1).  The result equals dkv_score's when
+ *       lse[b, hq, r] = ln( sum over keys i <= P + r of exp(q[b,hq,r] . k[b,hq/G,i] / sqrt(D)) )   (natural log).
+ *     lse : fp32 [Bt, Hq, ws], device, 4-byte aligned; finite.  Other arguments as for dkv_score.
+ * The library does not check lse against k: a wrong normaliser scales that row's contribution. */
+int dkv_score_lse(dkv_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* lse,
+                  float* scores_out, void* stream);
+
 /* Store caller-computed scores fp32 [Bt, Hkv, P] (finite, >= 0) as layer `layer` of the history,
  * in place of dkv_score (e.g. scores emitted by a fused prefill attention kernel). */
 int dkv_set_scores(dkv_ctx* ctx, int32_t layer, const float* scores, void* stream);

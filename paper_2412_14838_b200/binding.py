@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libdkv.so")
 
 EXPORTS = [
-    "dkv_create", "dkv_destroy", "dkv_reset", "dkv_score", "dkv_score_static", "dkv_set_scores", "dkv_select_topk", "dkv_rebudget",
+    "dkv_create", "dkv_destroy", "dkv_reset", "dkv_score", "dkv_score_static", "dkv_score_lse", "dkv_set_scores", "dkv_select_topk", "dkv_rebudget",
     "dkv_compact", "dkv_compact_all", "dkv_run_prefill_pass", "dkv_run_prefill_pass_host", "dkv_get_counts",
     "dkv_layer_views", "dkv_kept_sorted", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status", "dkv_profile", "dkv_profile_read", "dkv_launch_count", "dkv_last_cuda_error",
     "dkv_strerror", "dkv_version",
@@ -55,6 +55,7 @@ def load() -> ctypes.CDLL:
         "dkv_reset": [vp, vp],
         "dkv_score": [vp, i32, vp, vp, vp, vp],
         "dkv_score_static": [ctypes.POINTER(DkvConfig), vp, vp, vp, vp],
+        "dkv_score_lse": [vp, i32, vp, vp, vp, vp, vp],
         "dkv_set_scores": [vp, i32, vp, vp],
         "dkv_select_topk": [vp, i32, vp, vp, vp],
         "dkv_rebudget": [vp, i32, vp, vp],
@@ -165,6 +166,12 @@ def dkv_score_static(cfg: DkvConfig, q_win, k, scores_out, stream=None) -> None:
     """Score one layer without a context and without any device allocation (see include/dkv.h)."""
     _check(load().dkv_score_static(ctypes.byref(cfg), _ptr(q_win), _ptr(k), _ptr(scores_out), _stream(stream)),
            "dkv_score_static")
+
+
+def dkv_score_lse(ctx: int, layer: int, q_win, k, lse, scores_out=None, stream=None) -> None:
+    """Score one layer in a single sweep, given the window rows' log-sum-exp fp32 [Bt, Hq, ws] (see include/dkv.h)."""
+    _check(load().dkv_score_lse(ctx, layer, _ptr(q_win), _ptr(k), _ptr(lse), _ptr(scores_out), _stream(stream)),
+           "dkv_score_lse")
 
 
 def dkv_set_scores(ctx: int, layer: int, scores, stream=None) -> None:

@@ -197,6 +197,7 @@ bool make_job(dkv_ctx* c, int mode, int layer, const void* q, const void* k, flo
   p->mode = mode;
   p->out_scale = (c->cfg.flags & DKV_F_WINDOW_MEAN) ? 1.0f / (float)s.M : 1.0f;
   p->pool_avg = c->cfg.pool_kind == 1;
+  p->lse_in = nullptr;
   p->idesc = mode == tc::kStats ? make_idesc(128, 128) : make_idesc(128, p->nq16);
   return true;
 }
@@ -216,6 +217,23 @@ int launch_score(dkv_ctx* c, int stats_layer, const void* sq, const void* sk, in
   ProfScope ps(c, stats_layer >= 0 ? DKV_STEP_SCORE_STATS : DKV_STEP_SCORE_EMIT, 1, st);
   tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm0, km0, qm1, km1, j0, j1);
   DKV_LAUNCHED(c);
+  return DKV_OK;
+}
+
+// Sweep 2 alone, with the window rows' normalisers supplied by the caller instead of sweep 1.
+int do_score_lse(dkv_ctx* c, int layer, const void* q, const void* k, const float* lse, float* scores_out,
+                 cudaStream_t st) {
+  CUtensorMap qm, km;
+  tc::Params job, none;
+  memset(&job, 0, sizeof job); memset(&none, 0, sizeof none);
+  none.mode = tc::kNone;
+  if (!make_job(c, tc::kEmit, layer, q, k, scores_out, layer % 3, &qm, &km, &job)) return DKV_ERR_CUDA;
+  job.lse_in = lse;
+  ProfScope ps(c, DKV_STEP_SCORE_EMIT, 1, st);
+  tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, qm, km, job, none);
+  DKV_LAUNCHED(c);
+  c->scored[layer] = 1;
+  c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
   return DKV_OK;
 }
 
@@ -581,6 +599,15 @@ int dkv_score(dkv_ctx* c, int32_t layer, const void* q_win, const void* k, float
   return do_score(c, layer, q_win, k, scores_out, as_stream(stream));
 }
 
+int dkv_score_lse(dkv_ctx* c, int32_t layer, const void* q_win, const void* k, const float* lse, float* scores_out,
+                  void* stream) {
+  int rc = check_layer(c, layer);
+  if (rc) return rc;
+  if (!q_win || !k || !lse || !aligned16(q_win) || !aligned16(k) || !aligned16(scores_out) || ((uintptr_t)lse & 3))
+    return DKV_ERR_INVALID_ARG;
+  return do_score_lse(c, layer, q_win, k, lse, scores_out, as_stream(stream));
+}
+
 int dkv_set_scores(dkv_ctx* c, int32_t layer, const float* scores, void* stream) {
   int rc = check_layer(c, layer);
   if (rc) return rc;
@@ -820,6 +847,7 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   if (!make_map(&qm, q_win, D, M, heads) || !make_map(&km, k, D, S, heads)) return DKV_ERR_CUDA;
   if (cudaMemsetAsync(su.ptr, 0, 256, st) != cudaSuccess) return DKV_ERR_CUDA;   // status words start at zero
   tc::Params p, none;
+  memset(&p, 0, sizeof p);
   memset(&none, 0, sizeof none);
   none.mode = tc::kNone;
   p.S = S; p.P = P; p.ws = cfg->window; p.M = M; p.D = D; p.heads = heads; p.half = cfg->pool_kernel / 2;

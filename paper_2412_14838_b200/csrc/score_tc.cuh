@@ -58,6 +58,7 @@ struct Params {
   int mode;                // kNone: nothing to do
   float out_scale;         // sweep 2: factor on the raw scores before pooling (1, or 1/(ws*G) for the window mean)
   int pool_avg;            // sweep 2: 0 = max-pool, 1 = average over the neighbours that exist
+  const float* lse_in;     // sweep 2: caller's natural-log normalisers [heads][M] (then sweep 1 never ran), or null
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -433,7 +434,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
             const int c_lo = tile_owner((long long)sg.bh * p.tph, total, p.stats_grid);
             const int c_hi = tile_owner((long long)(sg.bh + 1) * p.tph - 1, total, p.stats_grid);
             float lse = INFINITY;
-            if (sid < p.M) {
+            if (p.lse_in) {
+              if (sid < p.M) lse = p.lse_in[(size_t)sg.bh * p.M + sid] * kLog2e;
+            } else if (sid < p.M) {
               float m = -INFINITY;
               for (int c = 0; c <= c_hi - c_lo; ++c) m = fmaxf(m, p.stats[((size_t)sg.bh * p.slots + c) * p.m_stride + sid].x);
               float l = 0.f;
