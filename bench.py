@@ -282,14 +282,19 @@ def run_gpu(args, w):
     B.dkv_profile(ctx, False)
     peaks, peak_kind = measured_peaks()
     peak = float(peaks["hbm_gbs"])
+    # the scoring kernel: every launch sweeps a group of layers (sweep 2 of one group, sweep 1 of the next), so
+    # the algorithmic bytes of a launch are the pass's K bytes over the launches of a pass
     score_ms = (prof["score_stats"][0] + prof["score_emit"][0] + prof["pool"][0]) / args.steps
-    score_launch_ms = score_ms / w.L                      # one layer's scoring = one "launch" of the scoring step
+    score_launches = (prof["score_stats"][1] + prof["score_emit"][1] + prof["pool"][1]) / args.steps
+    score_launch_ms = score_ms / score_launches
     k_bytes = w.k_bytes_per_layer()
-    achieved = k_bytes / (score_launch_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "window scoring (softmax statistics sweep + emit sweep + pooling), per layer",
+    launch_bytes = k_bytes * w.L / score_launches
+    achieved = launch_bytes / (score_launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "window scoring (softmax statistics sweep + emit sweep + pooling)",
                 "achieved": achieved, "peak": peak, "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})",
                 "unit": "GB/s", "frac": achieved / peak,
-                "algorithmic_bytes_per_launch": k_bytes, "avg_launch_ms": score_launch_ms,
+                "algorithmic_bytes_per_launch": launch_bytes, "avg_launch_ms": score_launch_ms,
+                "launches_per_pass": score_launches, "scoring_ms_per_layer": score_ms / w.L,
                 "traffic": (ncu_traffic(w) or {}).get("live_bytes_per_launch"),
                 "traffic_cold_cache": (ncu_traffic(w) or {}).get("cold_bytes_per_launch"),
                 "whole_pass": {"algorithmic_bytes": w.algorithmic_bytes(),

@@ -19,6 +19,8 @@ using namespace dkv;
 
 struct ProfRec { cudaEvent_t a, b; int step; int launches; };
 
+constexpr int kSideStreams = 4;
+
 struct dkv_ctx {
   dkv_config cfg;
   Shape s;
@@ -43,12 +45,14 @@ struct dkv_ctx {
   size_t sel_smem;
   // tensor-core scoring
   int n_sms, tc_grid, tc_slots;
-  float2* d_tc_stats;   // [3][Bt*Hkv][tc_slots][256]: partial softmax statistics, three layers in rotation
+  int pass_group;       // layers per scoring launch of dkv_run_prefill_pass (1..tc::kMaxGroup)
+  float2* d_tc_stats;   // [3][kMaxGroup*Bt*Hkv][tc_slots][256]: partial softmax statistics, three jobs in rotation
   cudaStream_t hi;      // scoring launches of dkv_run_prefill_pass: highest priority, so that a freed SM goes to a
                         // waiting scoring CTA before the side streams' many short CTAs
   cudaStream_t upd;     // budget updates (rebudget + shrink) of dkv_run_prefill_pass, off the select streams
-  cudaStream_t side[2]; // side streams of dkv_run_prefill_pass (select / gather / rebudget / shrink), layers alternate
-  cudaEvent_t ev_fork, ev_join[3], ev_update, ev_scored[DKV_MAX_LAYERS], ev_picked[DKV_MAX_LAYERS], ev_selected[DKV_MAX_LAYERS];
+  cudaStream_t side[kSideStreams]; // side streams of dkv_run_prefill_pass (select / gather), layers in rotation
+  int n_side;           // how many of them the pass uses
+  cudaEvent_t ev_fork, ev_join[kSideStreams + 1], ev_update, ev_scored[DKV_MAX_LAYERS], ev_picked[DKV_MAX_LAYERS], ev_selected[DKV_MAX_LAYERS];
   // host state
   uint8_t scored[DKV_MAX_LAYERS], selected[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
   long long launches;
@@ -177,19 +181,25 @@ uint32_t make_idesc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// Parameters of one sweep over one layer; `buf` picks the statistics scratch (layers alternate).
-bool make_job(dkv_ctx* c, int mode, int layer, const void* q, const void* k, float* scores_out, int buf,
-              CUtensorMap* qm, CUtensorMap* km, tc::Params* p) {
+// Parameters of one sweep over the `nl` consecutive layers that start at `layer` (q, k: their nl device
+// pointers); `buf` picks the statistics scratch (jobs in flight rotate).  Sweep 2 of a multi-layer job walks the
+// layers backwards: the one sweep 1 streamed last is still partly in L2.
+bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, const void* const* k, float* scores_out,
+              int buf, tc::Maps* maps, tc::Params* p) {
   const Shape& s = c->s;
   const int heads = s.Bt * s.Hkv;
-  if (!make_map(qm, q, s.D, s.M, heads) || !make_map(km, k, s.D, s.S, heads)) return false;
-  p->S = s.S; p->P = s.P; p->ws = s.ws; p->M = s.M; p->D = s.D; p->heads = heads; p->half = s.pool / 2;
+  for (int i = 0; i < tc::kMaxGroup; ++i) {
+    const int j = i < nl ? i : 0;                          // unused entries repeat the first (never read)
+    if (!make_map(&maps->q[i], q[j], s.D, s.M, heads) || !make_map(&maps->k[i], k[j], s.D, s.S, heads)) return false;
+  }
+  p->S = s.S; p->P = s.P; p->ws = s.ws; p->M = s.M; p->D = s.D; p->heads = nl * heads; p->half = s.pool / 2;
+  p->nl = nl; p->hpl = heads; p->rev = (mode == tc::kEmit && nl > 1) ? 1 : 0;
   p->tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
   p->nq16 = (s.M + 15) / 16 * 16;
   p->nmblk = (s.M + 127) / 128;
   p->slots = c->tc_slots; p->m_stride = 256;
   p->scale2 = kLog2e / sqrtf((float)s.D);
-  p->stats = c->d_tc_stats + (size_t)buf * heads * c->tc_slots * 256;
+  p->stats = c->d_tc_stats + (size_t)buf * tc::kMaxGroup * heads * c->tc_slots * 256;
   p->scores = c->d_scores + (size_t)layer * layer_scores(s);
   p->copy_out = scores_out;
   p->status = c->d_status;
@@ -202,20 +212,22 @@ bool make_job(dkv_ctx* c, int mode, int layer, const void* q, const void* k, flo
   return true;
 }
 
-// One launch: sweep 2 of `emit_layer` (if >= 0), then sweep 1 of `stats_layer` (if >= 0).  In the pass the
-// emit layer is the one whose keys the previous launch streamed last, so its second read finds them in L2.
-int launch_score(dkv_ctx* c, int stats_layer, const void* sq, const void* sk, int emit_layer, const void* eq,
-                 const void* ek, float* scores_out, cudaStream_t st) {
-  CUtensorMap qm0, km0, qm1, km1;
+// One launch: sweep 2 of the `en` layers from `emit_layer` (if >= 0), then sweep 1 of the `sn` layers from
+// `stats_layer` (if >= 0).  In the pass the emit layers are the ones the previous launch streamed, so their
+// second read finds the most recent of them in L2.  `sbuf`, `ebuf`: statistics scratch of either job.
+int launch_score(dkv_ctx* c, int stats_layer, int sn, const void* const* sq, const void* const* sk, int sbuf,
+                 int emit_layer, int en, const void* const* eq, const void* const* ek, int ebuf, float* scores_out,
+                 cudaStream_t st) {
+  tc::Maps m0, m1;
   tc::Params j0, j1;
   memset(&j0, 0, sizeof j0); memset(&j1, 0, sizeof j1);
   j0.mode = j1.mode = tc::kNone;
-  if (emit_layer >= 0 && !make_job(c, tc::kEmit, emit_layer, eq, ek, scores_out, emit_layer % 3, &qm0, &km0, &j0)) return DKV_ERR_CUDA;
-  if (stats_layer >= 0 && !make_job(c, tc::kStats, stats_layer, sq, sk, nullptr, stats_layer % 3, &qm1, &km1, &j1)) return DKV_ERR_CUDA;
-  if (emit_layer < 0) { qm0 = qm1; km0 = km1; }
-  if (stats_layer < 0) { qm1 = qm0; km1 = km0; }
+  if (emit_layer >= 0 && !make_job(c, tc::kEmit, emit_layer, en, eq, ek, scores_out, ebuf, &m0, &j0)) return DKV_ERR_CUDA;
+  if (stats_layer >= 0 && !make_job(c, tc::kStats, stats_layer, sn, sq, sk, nullptr, sbuf, &m1, &j1)) return DKV_ERR_CUDA;
+  if (emit_layer < 0) m0 = m1;
+  if (stats_layer < 0) m1 = m0;
   ProfScope ps(c, stats_layer >= 0 ? DKV_STEP_SCORE_STATS : DKV_STEP_SCORE_EMIT, 1, st);
-  tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm0, km0, qm1, km1, j0, j1);
+  tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(m0, m1, j0, j1);
   DKV_LAUNCHED(c);
   return DKV_OK;
 }
@@ -223,14 +235,14 @@ int launch_score(dkv_ctx* c, int stats_layer, const void* sq, const void* sk, in
 // Sweep 2 alone, with the window rows' normalisers supplied by the caller instead of sweep 1.
 int do_score_lse(dkv_ctx* c, int layer, const void* q, const void* k, const float* lse, float* scores_out,
                  cudaStream_t st) {
-  CUtensorMap qm, km;
+  tc::Maps maps;
   tc::Params job, none;
   memset(&job, 0, sizeof job); memset(&none, 0, sizeof none);
   none.mode = tc::kNone;
-  if (!make_job(c, tc::kEmit, layer, q, k, scores_out, layer % 3, &qm, &km, &job)) return DKV_ERR_CUDA;
+  if (!make_job(c, tc::kEmit, layer, 1, &q, &k, scores_out, layer % 3, &maps, &job)) return DKV_ERR_CUDA;
   job.lse_in = lse;
   ProfScope ps(c, DKV_STEP_SCORE_EMIT, 1, st);
-  tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, qm, km, job, none);
+  tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(maps, maps, job, none);
   DKV_LAUNCHED(c);
   c->scored[layer] = 1;
   c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
@@ -238,9 +250,9 @@ int do_score_lse(dkv_ctx* c, int layer, const void* q, const void* k, const floa
 }
 
 int do_score(dkv_ctx* c, int layer, const void* q, const void* k, float* scores_out, cudaStream_t st) {
-  int rc = launch_score(c, layer, q, k, -1, nullptr, nullptr, nullptr, st);
+  int rc = launch_score(c, layer, 1, &q, &k, layer % 3, -1, 0, nullptr, nullptr, 0, nullptr, st);
   if (rc) return rc;
-  if ((rc = launch_score(c, -1, nullptr, nullptr, layer, q, k, scores_out, st))) return rc;
+  if ((rc = launch_score(c, -1, 0, nullptr, nullptr, 0, layer, 1, &q, &k, layer % 3, scores_out, st))) return rc;
   c->scored[layer] = 1;
   c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
   return DKV_OK;
@@ -349,54 +361,67 @@ int do_reset(dkv_ctx* c, cudaStream_t st) {
   return DKV_OK;
 }
 
-// Algorithm 1's loop.  The scoring launches run back to back on `st` (launch l = sweep 1 of layer l
-// followed by sweep 2 of layer l-1); everything that consumes a layer's scores (select, gather, and
-// every m layers rebudget + shrink) runs on two side streams, layers alternating between them, behind
-// events, so that it overlaps the scoring of the following layers.  `st` rejoins both at the end.
+// Algorithm 1's loop.  The scoring launches run back to back on a stream of their own; launch g runs sweep 2
+// of layer group g-1 and then sweep 1 of group g (a group = up to `pass_group` consecutive layers, so that the
+// fixed cost of a launch and of a job is paid once per group).  Everything that consumes a layer's scores (select,
+// gather, and every m layers rebudget + shrink) runs on side streams behind events, layers alternating between
+// two of them, so that it overlaps the scoring of the following groups.  `st` rejoins all of them at the end.
 int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* const* v, void* const* kb,
             void* const* vb, cudaStream_t st) {
   const Shape& s = c->s;
   int rc = do_reset(c, st);
   if (rc) return rc;
   DKV_CUDA(c, cudaEventRecord(c->ev_fork, st));
-  for (int i = 0; i < 2; ++i) DKV_CUDA(c, cudaStreamWaitEvent(c->side[i], c->ev_fork, 0));
+  for (int i = 0; i < c->n_side; ++i) DKV_CUDA(c, cudaStreamWaitEvent(c->side[i], c->ev_fork, 0));
   DKV_CUDA(c, cudaStreamWaitEvent(c->hi, c->ev_fork, 0));
   DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_fork, 0));
   cudaStream_t caller = st;
   st = c->hi;
-  for (int l = 0; l <= s.L; ++l) {
-    const int sl = l < s.L ? l : -1, el = l - 1;
-    if ((rc = launch_score(c, sl, sl >= 0 ? q[sl] : nullptr, sl >= 0 ? k[sl] : nullptr, el, el >= 0 ? q[el] : nullptr,
-                           el >= 0 ? k[el] : nullptr, nullptr, st)))
+  // Group sizes: as large as allowed while many layers remain, halving towards the end, so that the work
+  // that can only start after the last launch (select, gather, update of the last group) is one layer's.
+  int first[DKV_MAX_LAYERS + 2], groups = 0;
+  for (int done = 0; done < s.L;) {
+    int n = (s.L - done) / 2;
+    if (n > c->pass_group) n = c->pass_group;
+    if (n < 1) n = 1;
+    first[groups++] = done;
+    done += n;
+  }
+  first[groups] = s.L;
+  for (int g = 0; g <= groups; ++g) {
+    const int sl = g < groups ? first[g] : -1, sn = g < groups ? first[g + 1] - first[g] : 0;
+    const int e0 = g > 0 ? first[g - 1] : -1, en = g > 0 ? first[g] - first[g - 1] : 0;
+    if ((rc = launch_score(c, sl, sn, sl >= 0 ? q + sl : nullptr, sl >= 0 ? k + sl : nullptr, g % 3, e0, en,
+                           e0 >= 0 ? q + e0 : nullptr, e0 >= 0 ? k + e0 : nullptr, (g + 2) % 3, nullptr, st)))
       return rc;
-    if (el < 0) continue;
-    c->scored[el] = 1;
-    cudaStream_t sd = c->side[el & 1];
-    DKV_CUDA(c, cudaEventRecord(c->ev_scored[el], st));
-    DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_scored[el], 0));
-    if ((rc = do_select(c, el, nullptr, nullptr, sd))) return rc;
-    DKV_CUDA(c, cudaEventRecord(c->ev_picked[el], sd));
-    if ((rc = do_gather(c, el, k[el], v[el], kb[el], vb[el], sd))) return rc;
-    DKV_CUDA(c, cudaEventRecord(c->ev_selected[el], sd));
-    const bool update = ((el + 1) % s.m == 0) || (el + 1 == s.L && s.L % s.m != 0);
-    if (update) {
-      // The rebudget needs every earlier layer selected (both select streams, each in layer order), the shrink
-      // also gathered; the previous update precedes it on the same stream.  Later layers' select and gather
-      // do not wait for it: an update changes the counts and buffers of the layers before it only.
-      DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_picked[el], 0));
-      if (el >= 1) DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_picked[el - 1], 0));
-      if ((rc = do_rebudget(c, el + 1, nullptr, c->upd))) return rc;
-      DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_selected[el], 0));
-      if (el >= 1) DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_selected[el - 1], 0));
-      if ((rc = do_shrink(c, 0, el + 1, kb, vb, c->upd))) return rc;
+    if (e0 < 0) continue;
+    DKV_CUDA(c, cudaEventRecord(c->ev_scored[e0], st));
+    for (int el = e0; el < e0 + en; ++el) {
+      c->scored[el] = 1;
+      cudaStream_t sd = c->side[el % c->n_side];
+      DKV_CUDA(c, cudaStreamWaitEvent(sd, c->ev_scored[e0], 0));
+      if ((rc = do_select(c, el, nullptr, nullptr, sd))) return rc;
+      DKV_CUDA(c, cudaEventRecord(c->ev_picked[el], sd));
+      if ((rc = do_gather(c, el, k[el], v[el], kb[el], vb[el], sd))) return rc;
+      DKV_CUDA(c, cudaEventRecord(c->ev_selected[el], sd));
+      const bool update = ((el + 1) % s.m == 0) || (el + 1 == s.L && s.L % s.m != 0);
+      if (update) {
+        // The rebudget needs every earlier layer selected (every select stream, each in layer order), the shrink
+        // also gathered; the previous update precedes it on the same stream.  Later layers' select and gather
+        // do not wait for it: an update changes the counts and buffers of the layers before it only.
+        for (int b = 0; b < c->n_side && b <= el; ++b) DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_picked[el - b], 0));
+        if ((rc = do_rebudget(c, el + 1, nullptr, c->upd))) return rc;
+        for (int b = 0; b < c->n_side && b <= el; ++b) DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_selected[el - b], 0));
+        if ((rc = do_shrink(c, 0, el + 1, kb, vb, c->upd))) return rc;
+      }
     }
   }
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < c->n_side; ++i) {
     DKV_CUDA(c, cudaEventRecord(c->ev_join[i], c->side[i]));
     DKV_CUDA(c, cudaStreamWaitEvent(caller, c->ev_join[i], 0));
   }
-  DKV_CUDA(c, cudaEventRecord(c->ev_join[2], c->hi));
-  DKV_CUDA(c, cudaStreamWaitEvent(caller, c->ev_join[2], 0));
+  DKV_CUDA(c, cudaEventRecord(c->ev_join[kSideStreams], c->hi));
+  DKV_CUDA(c, cudaStreamWaitEvent(caller, c->ev_join[kSideStreams], 0));
   DKV_CUDA(c, cudaEventRecord(c->ev_update, c->upd));
   DKV_CUDA(c, cudaStreamWaitEvent(caller, c->ev_update, 0));
   return DKV_OK;
@@ -407,7 +432,7 @@ void free_all(dkv_ctx* c) {
   cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_rb_state); cudaFree(c->d_rb_above); cudaFree(c->d_rb_hist1);
   cudaFree(c->d_rb_above2); cudaFree(c->d_rb_hist2); cudaFree(c->d_layer_hist);
   cudaFree(c->d_cand); cudaFree(c->d_cand_n); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
-  for (int i = 0; i < 2; ++i) if (c->side[i]) cudaStreamDestroy(c->side[i]);
+  for (int i = 0; i < kSideStreams; ++i) if (c->side[i]) cudaStreamDestroy(c->side[i]);
   if (c->hi) cudaStreamDestroy(c->hi);
   if (c->pass_exec) cudaGraphExecDestroy(c->pass_exec);
   delete c->pass_key;
@@ -415,7 +440,7 @@ void free_all(dkv_ctx* c) {
   if (c->ev_gfork) cudaEventDestroy(c->ev_gfork);
   if (c->ev_gjoin) cudaEventDestroy(c->ev_gjoin);
   if (c->upd) cudaStreamDestroy(c->upd);
-  for (int i = 0; i < 3; ++i) if (c->ev_join[i]) cudaEventDestroy(c->ev_join[i]);
+  for (int i = 0; i <= kSideStreams; ++i) if (c->ev_join[i]) cudaEventDestroy(c->ev_join[i]);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_update) cudaEventDestroy(c->ev_update);
   for (int l = 0; l < DKV_MAX_LAYERS; ++l) {
@@ -504,19 +529,29 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
     c->n_sms = sms > 0 ? sms : 1;
     const int tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
     const long long total_tiles = (long long)heads * tph;
-    // leave a few SMs to the per-head select CTAs that dkv_run_prefill_pass runs beside the scoring
-    int side = 2 * heads < c->n_sms / 6 ? 2 * heads : c->n_sms / 6;
+    // leave some SMs to the select / gather / update kernels that dkv_run_prefill_pass runs beside the scoring:
+    // with grouped launches up to four layers' selects (one CTA per head) are in flight at once
+    int side = 4 * heads < c->n_sms * 2 / 9 ? 4 * heads : c->n_sms * 2 / 9;
     if (const char* e = getenv("DKV_SIDE_SMS")) side = atoi(e);
     int score_sms = c->n_sms - side;
     if (score_sms < 1) score_sms = 1;
     c->tc_grid = (int)(total_tiles < score_sms ? total_tiles : score_sms);
     int slots = 1;
-    for (int bh = 0; bh < heads; ++bh) {
-      const int lo = tc::tile_owner((long long)bh * tph, total_tiles, c->tc_grid);
-      const int hi = tc::tile_owner((long long)(bh + 1) * tph - 1, total_tiles, c->tc_grid);
-      if (hi - lo + 1 > slots) slots = hi - lo + 1;
-    }
+    for (int nl = 1; nl <= tc::kMaxGroup; ++nl)           // a job may cover up to kMaxGroup layers (the pass groups them)
+      for (int bh = 0; bh < nl * heads; ++bh) {
+        const int lo = tc::tile_owner((long long)bh * tph, nl * total_tiles, c->tc_grid);
+        const int hi = tc::tile_owner((long long)(bh + 1) * tph - 1, nl * total_tiles, c->tc_grid);
+        if (hi - lo + 1 > slots) slots = hi - lo + 1;
+      }
     c->tc_slots = slots;
+    c->pass_group = 4;
+    if (const char* e = getenv("DKV_PASS_GROUP")) c->pass_group = atoi(e);
+    if (c->pass_group < 1) c->pass_group = 1;
+    if (c->pass_group > tc::kMaxGroup) c->pass_group = tc::kMaxGroup;
+    c->n_side = kSideStreams;
+    if (const char* e = getenv("DKV_SIDE_STREAMS")) c->n_side = atoi(e);
+    if (c->n_side < 1) c->n_side = 1;
+    if (c->n_side > kSideStreams) c->n_side = kSideStreams;
   }
   const size_t bl = (size_t)s.Bt * s.L;
 #define TRY(call) if (e == cudaSuccess) e = (call)
@@ -533,9 +568,9 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMalloc(&c->d_layer_hist, sizeof(unsigned int) * s.L * s.Bt * kBins));
   TRY(cudaMalloc(&c->d_cand, sizeof(uint2) * s.L * layer_scores(s)));
   TRY(cudaMalloc(&c->d_cand_n, sizeof(unsigned int) * s.Bt));
-  TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * 3 * heads * c->tc_slots * 256));
+  TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * 3 * tc::kMaxGroup * heads * c->tc_slots * 256));
   TRY(cudaFuncSetAttribute(tc::score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
-  for (int i = 0; i < 2; ++i) TRY(cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking));
+  for (int i = 0; i < kSideStreams; ++i) TRY(cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking));
   TRY(cudaStreamCreateWithFlags(&c->gstream, cudaStreamNonBlocking));
   TRY(cudaEventCreateWithFlags(&c->ev_gfork, cudaEventDisableTiming));
   TRY(cudaEventCreateWithFlags(&c->ev_gjoin, cudaEventDisableTiming));
@@ -548,7 +583,7 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
     TRY(cudaDeviceGetStreamPriorityRange(&least, &greatest));
     TRY(cudaStreamCreateWithPriority(&c->hi, cudaStreamNonBlocking, greatest));
   }
-  for (int i = 0; i < 3; ++i) TRY(cudaEventCreateWithFlags(&c->ev_join[i], cudaEventDisableTiming));
+  for (int i = 0; i <= kSideStreams; ++i) TRY(cudaEventCreateWithFlags(&c->ev_join[i], cudaEventDisableTiming));
   TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
   TRY(cudaEventCreateWithFlags(&c->ev_update, cudaEventDisableTiming));
   for (int l = 0; l < s.L; ++l) {
@@ -843,14 +878,16 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   const unsigned long long need = 256ull + (unsigned long long)heads * slots * 256ull * sizeof(float2);
   if (need > DKV_STATIC_SCRATCH_BYTES) return DKV_ERR_TOO_LARGE;
   cudaStream_t st = as_stream(stream);
-  CUtensorMap qm, km;
-  if (!make_map(&qm, q_win, D, M, heads) || !make_map(&km, k, D, S, heads)) return DKV_ERR_CUDA;
+  tc::Maps maps;
+  for (int i = 0; i < tc::kMaxGroup; ++i)
+    if (!make_map(&maps.q[i], q_win, D, M, heads) || !make_map(&maps.k[i], k, D, S, heads)) return DKV_ERR_CUDA;
   if (cudaMemsetAsync(su.ptr, 0, 256, st) != cudaSuccess) return DKV_ERR_CUDA;   // status words start at zero
   tc::Params p, none;
   memset(&p, 0, sizeof p);
   memset(&none, 0, sizeof none);
   none.mode = tc::kNone;
   p.S = S; p.P = P; p.ws = cfg->window; p.M = M; p.D = D; p.heads = heads; p.half = cfg->pool_kernel / 2;
+  p.nl = 1; p.hpl = heads; p.rev = 0;
   p.tph = tph; p.nq16 = (M + 15) / 16 * 16; p.nmblk = (M + 127) / 128;
   p.slots = slots; p.m_stride = 256;
   p.scale2 = kLog2e / sqrtf((float)D);
@@ -862,11 +899,11 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   p.stats_grid = grid;
   p.mode = tc::kStats;
   p.idesc = make_idesc(128, 128);
-  tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, qm, km, p, none);
+  tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(maps, maps, p, none);
   if (cudaPeekAtLastError() != cudaSuccess) return DKV_ERR_CUDA;
   p.mode = tc::kEmit;
   p.idesc = make_idesc(128, p.nq16);
-  tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(qm, km, qm, km, none, p);
+  tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(maps, maps, none, p);
   if (cudaPeekAtLastError() != cudaSuccess) return DKV_ERR_CUDA;
   return DKV_OK;
 }

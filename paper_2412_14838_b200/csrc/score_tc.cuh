@@ -59,7 +59,21 @@ struct Params {
   float out_scale;         // sweep 2: factor on the raw scores before pooling (1, or 1/(ws*G) for the window mean)
   int pool_avg;            // sweep 2: 0 = max-pool, 1 = average over the neighbours that exist
   const float* lse_in;     // sweep 2: caller's natural-log normalisers [heads][M] (then sweep 1 never ran), or null
+  int nl;                  // layers this job covers (1..kMaxGroup); `heads` counts the heads of all of them
+  int hpl;                 // heads per layer
+  int rev;                 // 1: the job walks its layers from the last to the first (sweep 2 after a grouped sweep 1:
+                           // the layer streamed last is the one most of whose keys are still in L2)
 };
+
+constexpr int kMaxGroup = 8;               // layers one job may cover
+struct Maps {                              // tensor maps of a job's layers, in storage order
+  CUtensorMap q[kMaxGroup], k[kMaxGroup];
+};
+
+// Head index in storage order (layer-major) of the head a job visits as number `bh`.
+__device__ __forceinline__ int stored_head(const Params& p, int bh) {
+  return p.rev ? (p.nl - 1 - bh / p.hpl) * p.hpl + bh % p.hpl : bh;
+}
 
 // ------------------------------------------------------------------------------------------ PTX
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -203,10 +217,9 @@ __host__ __device__ __forceinline__ int tile_owner(long long x, long long total,
 }
 
 // ------------------------------------------------------------------------------------------ kernel
-// job0 uses (q_map0, k_map0), job1 uses (q_map1, k_map1); a job with mode kNone is skipped.
+// job0 uses maps0, job1 uses maps1; a job with mode kNone is skipped.
 __global__ void __launch_bounds__(kThreads, 1)
-score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constant__ CUtensorMap k_map0,
-                const __grid_constant__ CUtensorMap q_map1, const __grid_constant__ CUtensorMap k_map1,
+score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps maps1,
                 const __grid_constant__ Params job0, const __grid_constant__ Params job1) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -252,13 +265,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
       for (int jb = 0; jb < 2; ++jb) {
         const Params& p = jb ? job1 : job0;
         if (p.mode == kNone) continue;
-        const CUtensorMap* q_map = jb ? &q_map1 : &q_map0;
-        const CUtensorMap* k_map = jb ? &k_map1 : &k_map0;
+        const Maps& maps = jb ? maps1 : maps0;
         const int halves = p.D / 64;
         const uint32_t tile_bytes = (uint32_t)halves * kHalfBytes;
         SegIter it(p, blockIdx.x, gridDim.x);
         Seg sg;
         while (it.next(sg)) {
+          const int nb = stored_head(p, sg.bh), hh = nb % p.hpl;
+          const CUtensorMap* q_map = &maps.q[nb / p.hpl];
+          const CUtensorMap* k_map = &maps.k[nb / p.hpl];
           if (sg.new_head) {
             // every MMA that read the previous queries must have finished: the last tile of either issuer
             for (int last = tile - 1; last >= 0 && last >= tile - 2; --last)
@@ -267,7 +282,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
               mbar_expect_tx(QFULL, (uint32_t)(p.nmblk * halves) * kHalfBytes);
               for (int h = 0; h < halves; ++h)
                 for (int mb = 0; mb < p.nmblk; ++mb)
-                  tma_load_3d(smem_u32(q_smem + h * (2 * kHalfBytes) + mb * kHalfBytes), q_map, QFULL, 64 * h, 128 * mb, sg.bh);
+                  tma_load_3d(smem_u32(q_smem + h * (2 * kHalfBytes) + mb * kHalfBytes), q_map, QFULL, 64 * h, 128 * mb, hh);
             }
           }
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
@@ -276,7 +291,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
             if (*abort_flag) break;
             mbar_expect_tx(FULL(s), tile_bytes);
             for (int h = 0; h < halves; ++h)
-              tma_load_3d(smem_u32(k_smem + (s * 2 + h) * kHalfBytes), k_map, FULL(s), 64 * h, sg.key0 + i * kTileKeys, sg.bh);
+              tma_load_3d(smem_u32(k_smem + (s * 2 + h) * kHalfBytes), k_map, FULL(s), 64 * h, sg.key0 + i * kTileKeys, hh);
           }
           if (*abort_flag) break;
         }
@@ -428,20 +443,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
           asm volatile("bar.sync 1, 512;" ::: "memory");
         } else {
           // ------------------------------------------------------------ sweep 2: one thread per key
+          const int nb = stored_head(p, sg.bh);              // sweep 1 filed its statistics in storage order
           if (sg.new_head && sid < 256) {
             // lse2 of every window row from the partial statistics of sweep 1
             const long long total = (long long)p.heads * p.tph;
-            const int c_lo = tile_owner((long long)sg.bh * p.tph, total, p.stats_grid);
-            const int c_hi = tile_owner((long long)(sg.bh + 1) * p.tph - 1, total, p.stats_grid);
+            const int c_lo = tile_owner((long long)nb * p.tph, total, p.stats_grid);
+            const int c_hi = tile_owner((long long)(nb + 1) * p.tph - 1, total, p.stats_grid);
             float lse = INFINITY;
             if (p.lse_in) {
-              if (sid < p.M) lse = p.lse_in[(size_t)sg.bh * p.M + sid] * kLog2e;
+              if (sid < p.M) lse = p.lse_in[(size_t)nb * p.M + sid] * kLog2e;
             } else if (sid < p.M) {
               float m = -INFINITY;
-              for (int c = 0; c <= c_hi - c_lo; ++c) m = fmaxf(m, p.stats[((size_t)sg.bh * p.slots + c) * p.m_stride + sid].x);
+              for (int c = 0; c <= c_hi - c_lo; ++c) m = fmaxf(m, p.stats[((size_t)nb * p.slots + c) * p.m_stride + sid].x);
               float l = 0.f;
               for (int c = 0; c <= c_hi - c_lo; ++c) {
-                const float2 st = p.stats[((size_t)sg.bh * p.slots + c) * p.m_stride + sid];
+                const float2 st = p.stats[((size_t)nb * p.slots + c) * p.m_stride + sid];
                 l += st.y * fast_exp2(st.x - m);
               }
               lse = m + log2f(l);
@@ -519,7 +535,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map0, const __grid_constan
                 if (o + d < p.P) v = fmaxf(v, raw_s[x + d]);
               }
             }
-            const size_t at = (size_t)sg.bh * p.P + o;
+            const size_t at = (size_t)nb * p.P + o;
             p.scores[at] = v;
             if (p.copy_out) p.copy_out[at] = v;
           }
