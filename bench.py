@@ -32,21 +32,23 @@ UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "mistral32k"
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM traffic of one scoring launch (dram__bytes_read.sum + dram__bytes_write.sum), taken with ncu on the
-# 4-layer cut of the mistral32k shape (same per-layer shape, so the figure needs no scaling; see
-# profiles/score_tc_kernel_mistral32k_4layers.md).  "live" is a single-pass capture without ncu's cache flush,
-# i.e. with whatever the previous launch left in L2, as in a real pass; "cold" is the --set full capture, where
-# every replay starts from flushed caches.  Both hold for the kernel source they were measured on and for that
-# per-layer shape only: any other source hash or shape reports null.
+# DRAM traffic of one full scoring launch (dram__bytes_read.sum + dram__bytes_write.sum): sweep 2 of four layers
+# followed by sweep 1 of the next four, taken with ncu on the 8-layer cut of the mistral32k shape (same per-layer
+# shape and group size, so the figure needs no scaling; see profiles/score_tc_kernel_mistral32k_8layers.md).
+# "live" is a single-pass capture without ncu's cache flush, i.e. with whatever the previous launch left in L2, as
+# in a real pass; "cold" is the --set full capture, where every replay starts from flushed caches.  Both hold for
+# the kernel source they were measured on, for that per-layer shape and for four-layer groups only: any other
+# source hash, shape or grouping reports null.
 NCU_TRAFFIC = {
-    "kernel_sha256": "f3ebfc768f27dfa9d6af7f839f8753d7e2be972a44665d7b5208e04b690248e7",
+    "kernel_sha256": "64ab6b981fecbf63f75af2617687efeb80d7c4d41e4feb6b33f82a4583b62cc3",
     "shape": (8, 128, 1, 32768, 32),          # Hkv, D, Bt, S, ws
-    "live_bytes_per_launch": 76_640_000 + 10_230_000,
-    "cold_bytes_per_launch": 134_960_000 + 4_050_000,
+    "layers_per_launch": 4,
+    "live_bytes_per_launch": 541_429_504 + 5_170_688,
+    "cold_bytes_per_launch": 542_036_480 + 8_006_144,
 }
 
 
-def ncu_traffic(w):
+def ncu_traffic(w, score_launches=None):
     import hashlib
     src = os.path.join(ROOT, "paper_2412_14838_b200", "csrc", "score_tc.cuh")
     try:
@@ -56,6 +58,9 @@ def ncu_traffic(w):
         return None
     if sha != NCU_TRAFFIC["kernel_sha256"] or (w.Hkv, w.D, w.Bt, w.S, w.ws) != NCU_TRAFFIC["shape"]:
         return None
+    g = NCU_TRAFFIC["layers_per_launch"]
+    if w.L % g or score_launches is None or round(score_launches) != w.L // g + 1:
+        return None                             # the pass was not run in full four-layer groups
     return NCU_TRAFFIC
 FALLBACK_HBM_GBS = 6650.0
 
@@ -295,8 +300,10 @@ def run_gpu(args, w):
                 "unit": "GB/s", "frac": achieved / peak,
                 "algorithmic_bytes_per_launch": launch_bytes, "avg_launch_ms": score_launch_ms,
                 "launches_per_pass": score_launches, "scoring_ms_per_layer": score_ms / w.L,
-                "traffic": (ncu_traffic(w) or {}).get("live_bytes_per_launch"),
-                "traffic_cold_cache": (ncu_traffic(w) or {}).get("cold_bytes_per_launch"),
+                "traffic": (ncu_traffic(w, score_launches) or {}).get("live_bytes_per_launch"),
+                "traffic_cold_cache": (ncu_traffic(w, score_launches) or {}).get("cold_bytes_per_launch"),
+                "traffic_note": "DRAM bytes of a full launch (sweep 2 of 4 layers + sweep 1 of the next 4); the first "
+                                "and last launch of a pass run one sweep only, so avg launches carry 8/9 of that",
                 "whole_pass": {"algorithmic_bytes": w.algorithmic_bytes(),
                                "achieved_gbs": w.algorithmic_bytes() / (ms_per_step * 1e-3) / 1e9,
                                "frac_of_measured_peak": w.algorithmic_bytes() / (ms_per_step * 1e-3) / 1e9 / peak,

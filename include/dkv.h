@@ -174,6 +174,9 @@ int dkv_compact_all(dkv_ctx* ctx, int32_t upto_layer, void* const* kb, void* con
 /* Algorithm 1's loop over all L layers: score, select, gather each layer; after every m-th layer (and
  * after the last one if L % m != 0) rebudget and shrink all preceding layers.  Resets the context first.
  * q_win, k, v, kb, vb : HOST arrays of L device pointers (layouts as above).
+ * All layers' tensors must be resident when the call is made: the scoring kernel is launched once per group of
+ * consecutive layers (sweep 2 of one group, sweep 1 of the next), the steps that consume a layer's scores run
+ * beside the following groups' scoring.  The results are those of the layer-by-layer loop.
  * The first call with a given set of pointers records the whole pass as a CUDA graph (on an internal stream
  * that forks from `stream` and rejoins it); later calls with the same pointers replay it, whatever the
  * buffers then contain.  The plain sequence of launches is used instead while dkv_profile is on, when

@@ -45,6 +45,7 @@ struct dkv_ctx {
   size_t sel_smem;
   // tensor-core scoring
   int n_sms, tc_grid, tc_slots;
+  int pass_taper;       // group sizes halve towards the end of the pass
   int pass_group;       // layers per scoring launch of dkv_run_prefill_pass (1..tc::kMaxGroup)
   float2* d_tc_stats;   // [3][kMaxGroup*Bt*Hkv][tc_slots][256]: partial softmax statistics, three jobs in rotation
   cudaStream_t hi;      // scoring launches of dkv_run_prefill_pass: highest priority, so that a freed SM goes to a
@@ -377,12 +378,13 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
   DKV_CUDA(c, cudaStreamWaitEvent(c->upd, c->ev_fork, 0));
   cudaStream_t caller = st;
   st = c->hi;
-  // Group sizes: as large as allowed while many layers remain, halving towards the end, so that the work
-  // that can only start after the last launch (select, gather, update of the last group) is one layer's.
+  // Group sizes: `pass_group` layers each.  (With DKV_PASS_TAPER=1 they halve towards the end, so that less work
+  // is left for after the last launch; with four select streams that tail is as short either way.)
   int first[DKV_MAX_LAYERS + 2], groups = 0;
   for (int done = 0; done < s.L;) {
-    int n = (s.L - done) / 2;
+    int n = c->pass_taper ? (s.L - done) / 2 : c->pass_group;
     if (n > c->pass_group) n = c->pass_group;
+    if (n > s.L - done) n = s.L - done;
     if (n < 1) n = 1;
     first[groups++] = done;
     done += n;
@@ -544,11 +546,14 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
         if (hi - lo + 1 > slots) slots = hi - lo + 1;
       }
     c->tc_slots = slots;
-    c->pass_group = 4;
+    // layers per scoring launch of the pass: enough that a CTA's share of a job is some tens of tiles
+    c->pass_group = total_tiles / c->tc_grid < 8 ? tc::kMaxGroup : 4;
     if (const char* e = getenv("DKV_PASS_GROUP")) c->pass_group = atoi(e);
     if (c->pass_group < 1) c->pass_group = 1;
     if (c->pass_group > tc::kMaxGroup) c->pass_group = tc::kMaxGroup;
     c->n_side = kSideStreams;
+    c->pass_taper = 0;
+    if (const char* e = getenv("DKV_PASS_TAPER")) c->pass_taper = atoi(e);
     if (const char* e = getenv("DKV_SIDE_STREAMS")) c->n_side = atoi(e);
     if (c->n_side < 1) c->n_side = 1;
     if (c->n_side > kSideStreams) c->n_side = kSideStreams;

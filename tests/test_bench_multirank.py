@@ -63,9 +63,11 @@ def test_ncu_traffic_is_tied_to_kernel_source_and_shape(monkeypatch):
     import bench
     from paper_2412_14838_b200 import synth
     w = synth.WORKLOADS["mistral32k"]
-    got = bench.ncu_traffic(w)
+    got = bench.ncu_traffic(w, w.L // 4 + 1)
     if got is not None:                       # the source is the measured one
-        assert got["cold_bytes_per_launch"] >= got["live_bytes_per_launch"] >= w.k_bytes_per_layer()
-    assert bench.ncu_traffic(synth.WORKLOADS["tiny"]) is None
-    monkeypatch.setitem(bench.NCU_TRAFFIC, "kernel_sha256", "0" * 64)
+        assert got["cold_bytes_per_launch"] >= got["live_bytes_per_launch"] >= 4 * w.k_bytes_per_layer()
+    assert bench.ncu_traffic(w, w.L + 1) is None          # another grouping of the layers
     assert bench.ncu_traffic(w) is None
+    assert bench.ncu_traffic(synth.WORKLOADS["tiny"], 2) is None
+    monkeypatch.setitem(bench.NCU_TRAFFIC, "kernel_sha256", "0" * 64)
+    assert bench.ncu_traffic(w, w.L // 4 + 1) is None

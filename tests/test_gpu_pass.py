@@ -170,6 +170,28 @@ def test_pass_with_ragged_shape_and_final_partial_block():
         g.close()
 
 
+@pytest.mark.parametrize("group,taper,streams", [(1, 0, 1), (3, 0, 2), (8, 0, 4), (4, 1, 3)])
+def test_pass_is_the_same_however_the_layers_are_grouped(group, taper, streams, monkeypatch):
+    # The pass scores several layers per launch; the group size, a ragged last group, update points that fall
+    # inside a group (m = 2 with groups of 3) and the number of select streams are scheduling only.
+    monkeypatch.setenv("DKV_PASS_GROUP", str(group))
+    monkeypatch.setenv("DKV_PASS_TAPER", str(taper))
+    monkeypatch.setenv("DKV_SIDE_STREAMS", str(streams))
+    w = synth.Workload("grouppass", 52, L=7, Hq=8, Hkv=2, D=128, Bt=2, S=2100, ws=8, pool=5, N=24, Bl=64, m=2,
+                       recipe="sink")
+    g = GpuPass(w).run()            # the context reads the overrides when it is created
+    try:
+        check_properties(g)
+        compare_full(g)
+        B.dkv_run_prefill_pass(g.h, g.q, g.k, g.v, g.kb, g.vb)      # the replayed graph gives the same again
+        torch.cuda.synchronize()
+        again = np.zeros_like(g.counts)
+        B.dkv_get_counts(g.h, again)
+        assert (again == g.counts).all()
+    finally:
+        g.close()
+
+
 FULL = ["mistral32k", "llama16k_b4", "needle32k", "qwen16k"]
 
 
