@@ -179,7 +179,7 @@ class ClockSampler:
             except Exception as e:
                 self.err = repr(e)
                 return
-            time.sleep(0.02)
+            time.sleep(0.005)
 
     def __enter__(self):
         if self.err is None:
@@ -280,8 +280,9 @@ def run_gpu(args, w):
     value = whole_job_value(tokens, world, ms_per_step * 1e-3)
 
     # per-kernel durations: the same steps again, each step's launches bracketed by CUDA events
+    prof_steps = min(args.steps, 20)
     B.dkv_profile(ctx, True)
-    for _ in range(args.steps):
+    for _ in range(prof_steps):
         one_pass()
     prof = B.dkv_profile_read(ctx)
     B.dkv_profile(ctx, False)
@@ -289,8 +290,8 @@ def run_gpu(args, w):
     peak = float(peaks["hbm_gbs"])
     # the scoring kernel: every launch sweeps a group of layers (sweep 2 of one group, sweep 1 of the next), so
     # the algorithmic bytes of a launch are the pass's K bytes over the launches of a pass
-    score_ms = (prof["score_stats"][0] + prof["score_emit"][0] + prof["pool"][0]) / args.steps
-    score_launches = (prof["score_stats"][1] + prof["score_emit"][1] + prof["pool"][1]) / args.steps
+    score_ms = (prof["score_stats"][0] + prof["score_emit"][0] + prof["pool"][0]) / prof_steps
+    score_launches = (prof["score_stats"][1] + prof["score_emit"][1] + prof["pool"][1]) / prof_steps
     score_launch_ms = score_ms / score_launches
     k_bytes = w.k_bytes_per_layer()
     launch_bytes = k_bytes * w.L / score_launches
@@ -308,7 +309,7 @@ def run_gpu(args, w):
                                "achieved_gbs": w.algorithmic_bytes() / (ms_per_step * 1e-3) / 1e9,
                                "frac_of_measured_peak": w.algorithmic_bytes() / (ms_per_step * 1e-3) / 1e9 / peak,
                                "frac_of_8TBs": w.algorithmic_bytes() / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
-                "step_ms_per_pass": {n: round(t / args.steps, 4) for n, (t, _) in prof.items() if t > 0}}
+                "step_ms_per_pass": {n: round(t / prof_steps, 4) for n, (t, _) in prof.items() if t > 0}}
 
     # the one-sweep scoring entry point (normalisers given, as a prefill attention kernel would hand them over):
     # reported beside the headline, never part of it.  The normalisers are prepared outside the timed region.
@@ -327,12 +328,12 @@ def run_gpu(args, w):
             B.dkv_score_lse(ctx, l, q[l], k[l], lse[l], None, stream)
         barrier()
         ev0.record(stream)
-        for _ in range(args.steps):
+        for _ in range(prof_steps):
             for l in range(w.L):
                 B.dkv_score_lse(ctx, l, q[l], k[l], lse[l], None, stream)
         ev1.record(stream)
         barrier()
-        one_ms = max_over_ranks(ev0.elapsed_time(ev1)) / (args.steps * w.L)
+        one_ms = max_over_ranks(ev0.elapsed_time(ev1)) / (prof_steps * w.L)
         one_sweep = {"api": "dkv_score_lse", "avg_launch_ms": one_ms, "algorithmic_bytes_per_launch": k_bytes,
                      "achieved": k_bytes / (one_ms * 1e-3) / 1e9, "unit": "GB/s",
                      "frac": k_bytes / (one_ms * 1e-3) / 1e9 / peak}
@@ -379,7 +380,7 @@ def run_gpu(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="dkv", choices=["dkv", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))

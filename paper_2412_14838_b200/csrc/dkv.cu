@@ -184,7 +184,8 @@ uint32_t make_idesc(int M, int N) {
 
 // Parameters of one sweep over the `nl` consecutive layers that start at `layer` (q, k: their nl device
 // pointers); `buf` picks the statistics scratch (jobs in flight rotate).  Sweep 2 of a multi-layer job walks the
-// layers backwards: the one sweep 1 streamed last is still partly in L2.
+// layers backwards, starting with the one sweep 1 streamed last (with groups of several layers the counters show
+// no L2 hits from it: the group is larger than the cache).
 bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, const void* const* k, float* scores_out,
               int buf, tc::Maps* maps, tc::Params* p) {
   const Shape& s = c->s;
@@ -214,8 +215,7 @@ bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, con
 }
 
 // One launch: sweep 2 of the `en` layers from `emit_layer` (if >= 0), then sweep 1 of the `sn` layers from
-// `stats_layer` (if >= 0).  In the pass the emit layers are the ones the previous launch streamed, so their
-// second read finds the most recent of them in L2.  `sbuf`, `ebuf`: statistics scratch of either job.
+// `stats_layer` (if >= 0).  In the pass the emit layers are the ones the previous launch streamed.  `sbuf`, `ebuf`: statistics scratch of either job.
 int launch_score(dkv_ctx* c, int stats_layer, int sn, const void* const* sq, const void* const* sk, int sbuf,
                  int emit_layer, int en, const void* const* eq, const void* const* ek, int ebuf, float* scores_out,
                  cudaStream_t st) {
