@@ -183,9 +183,9 @@ uint32_t make_idesc(int M, int N) {
 }
 
 // Parameters of one sweep over the `nl` consecutive layers that start at `layer` (q, k: their nl device
-// pointers); `buf` picks the statistics scratch (jobs in flight rotate).  Sweep 2 of a multi-layer job walks the
-// layers backwards, starting with the one sweep 1 streamed last (with groups of several layers the counters show
-// no L2 hits from it: the group is larger than the cache).
+// pointers); `buf` picks the statistics scratch (jobs in flight rotate).  In sweep 2 every CTA walks its slice of the
+// key space from the end to the start: sweep 1 cut the same space into the same slices, so each CTA begins with
+// the keys that were streamed last and may still be in L2.
 bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, const void* const* k, float* scores_out,
               int buf, tc::Maps* maps, tc::Params* p) {
   const Shape& s = c->s;
@@ -195,7 +195,8 @@ bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, con
     if (!make_map(&maps->q[i], q[j], s.D, s.M, heads) || !make_map(&maps->k[i], k[j], s.D, s.S, heads)) return false;
   }
   p->S = s.S; p->P = s.P; p->ws = s.ws; p->M = s.M; p->D = s.D; p->heads = nl * heads; p->half = s.pool / 2;
-  p->nl = nl; p->hpl = heads; p->rev = (mode == tc::kEmit && nl > 1) ? 1 : 0;
+  p->nl = nl; p->hpl = heads; p->rev = 0;
+  p->back = (mode == tc::kEmit && !getenv("DKV_EMIT_FORWARD")) ? 1 : 0;
   p->tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
   p->nq16 = (s.M + 15) / 16 * 16;
   p->nmblk = (s.M + 127) / 128;

@@ -61,8 +61,9 @@ struct Params {
   const float* lse_in;     // sweep 2: caller's natural-log normalisers [heads][M] (then sweep 1 never ran), or null
   int nl;                  // layers this job covers (1..kMaxGroup); `heads` counts the heads of all of them
   int hpl;                 // heads per layer
-  int rev;                 // 1: the job walks its layers from the last to the first (sweep 2 after a grouped sweep 1:
-                           // the layer streamed last is the one most of whose keys are still in L2)
+  int rev;                 // 1: the job walks its layers from the last to the first
+  int back;                // sweep 2: 1 = every CTA walks its slice from the end to the start, so that it begins
+                           // with the keys sweep 1 streamed last (those still in L2)
 };
 
 constexpr int kMaxGroup = 8;               // layers one job may cover
@@ -180,9 +181,10 @@ struct Seg {
 
 struct SegIter {
   long long u, u_end;
-  int uph, half, cur_bh, mode;
+  int uph, half, cur_bh, mode, back;
   __device__ SegIter(const Params& p, int cta, int grid) {
     mode = p.mode;
+    back = p.mode == kEmit && p.back;
     uph = mode == kStats ? p.tph : p.P;
     const long long total = (long long)p.heads * uph;
     u = total * cta / grid;
@@ -192,6 +194,22 @@ struct SegIter {
   }
   __device__ bool next(Seg& s) {
     if (u >= u_end) return false;
+    if (back) {
+      // the last segment of what is left: it ends at u_end and starts at the head's first position, the
+      // slice's start or one segment's length before its end, whichever comes last
+      const int bh = (int)((u_end - 1) / uph);
+      long long b = (long long)bh * uph;
+      if (b < u) b = u;
+      if (b < u_end - (kMaxSegTiles * kTileKeys - 2 * half)) b = u_end - (kMaxSegTiles * kTileKeys - 2 * half);
+      const int off = (int)(b - (long long)bh * uph), len = (int)(u_end - b);
+      s.bh = bh;
+      s.out0 = off; s.out1 = off + len; s.key0 = off - half;
+      s.ntiles = (len + 2 * half + kTileKeys - 1) / kTileKeys;
+      s.new_head = bh != cur_bh;
+      cur_bh = bh;
+      u_end = b;
+      return true;
+    }
     const int bh = (int)(u / uph), off = (int)(u % uph);
     long long e = (long long)(bh + 1) * uph;
     if (e > u_end) e = u_end;
