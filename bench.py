@@ -290,8 +290,8 @@ def run_gpu(args, w):
     peak = float(peaks["hbm_gbs"])
     # the scoring kernel: every launch sweeps a group of layers (sweep 2 of one group, sweep 1 of the next), so
     # the algorithmic bytes of a launch are the pass's K bytes over the launches of a pass
-    score_ms = (prof["score_stats"][0] + prof["score_emit"][0] + prof["pool"][0]) / prof_steps
-    score_launches = (prof["score_stats"][1] + prof["score_emit"][1] + prof["pool"][1]) / prof_steps
+    score_ms = (prof["score_stats"][0] + prof["score_emit"][0]) / prof_steps
+    score_launches = (prof["score_stats"][1] + prof["score_emit"][1]) / prof_steps
     score_launch_ms = score_ms / score_launches
     k_bytes = w.k_bytes_per_layer()
     launch_bytes = k_bytes * w.L / score_launches

@@ -113,7 +113,11 @@ int dkv_score(dkv_ctx* ctx, int32_t layer, const void* q_win, const void* k, flo
  * 0.3 MB for 8 heads and 2 MB for 512 heads on a 148-SM part.
  *
  * The first call on each device looks up the array's device address and sets the kernels' shared
- * memory attribute (host-side, once).  Make that first call before starting any stream capture.
+ * memory attribute (host-side, once).  Make that first call before starting any stream capture, and
+ * before the caller's own pool takes the rest of the device memory: with CUDA's default lazy module
+ * loading the library image, and with it this array, is placed on the device at the first use of one of
+ * its kernels or symbols, i.e. inside that first call (CUDA_MODULE_LOADING=EAGER moves it to load time).
+ * A wait inside the kernels that runs out (see dkv_last_status) is reported by dkv_static_last_status.
  * All calls on a device share the one array, and it keeps whatever the last call left: the call
  * clears the status words it needs zeroed and overwrites every statistic before reading it, so
  * calls that follow one another on a stream are independent.  Calls that can overlap on the GPU
@@ -208,19 +212,37 @@ int dkv_budget_views(dkv_ctx* ctx, const int32_t** cnt, const int32_t** z, const
  * synchronise `stream`. */
 int dkv_memcpy_to_host(dkv_ctx* ctx, void* host_dst, const void* dev_src, uint64_t bytes, void* stream);
 /* Copy the status words to host int32 [8] (synchronises the device):
- * [0] first device-side error (0 = none), [1] kernels launched since dkv_create (host counter). */
+ * [0] first device-side failure since the last report (0 = none; else the number, 101..107, of the wait in
+ *     the scoring kernel that ran out first), [1] kernels launched since dkv_create (host counter),
+ * [2] the thread block of that wait.
+ * Returns DKV_OK when [0] is 0, else DKV_ERR_TIMEOUT: some wait inside a scoring launch since the last
+ * report gave up, and the scores of the layers scored since then are not to be used.  The kernel itself
+ * ended normally (no trap; its copies drained, its tensor memory freed), the context stays usable, and the
+ * failure is reported once: the device words are cleared by the call that reports it. */
 int dkv_last_status(dkv_ctx* ctx, int32_t* host_status);
+/* The same for dkv_score_static, whose status words live in the library's static scratch: host int32 [8] as
+ * above ([1] is 0).  Synchronises the current device; DKV_OK or DKV_ERR_TIMEOUT.  The next dkv_score_static
+ * call clears the words. */
+int dkv_static_last_status(int32_t* host_status);
+/* Limit of every wait inside the scoring kernel, in SM clock ticks (default 4e9, about 2 s; at least 1000).
+ * A wait that runs out makes its thread block stop issuing work, finish, and record the failure for
+ * dkv_last_status.  Applies to launches made after the call. */
+int dkv_set_wait_limit(dkv_ctx* ctx, int64_t clock_ticks);
+/* Test hook for the path above: in the launches that follow, thread block 0 never loads its key tile number
+ * `tile` (0-based, per launch) of scoring sweep `sweep` (1 = statistics, 2 = emit), so the wait for that
+ * tile runs out after the wait limit.  tile < 0 switches the hook off.  Nothing else is disturbed: no
+ * invalid address, no trap. */
+int dkv_debug_withhold_tile(dkv_ctx* ctx, int32_t sweep, int32_t tile);
 /* Optional per-step timing.  While enabled, every step's launches are bracketed by a pair of CUDA
  * events on the step's stream.  dkv_profile_read synchronises the device and returns, per step
  * (DKV_STEP_*), the summed event time in milliseconds and the number of kernels covered since the
  * last read, then clears the sums.  ms, launches : host arrays of DKV_N_STEPS entries. */
 #define DKV_STEP_SCORE_STATS 0   /* sweep 1 of the scoring: softmax statistics per window row */
-#define DKV_STEP_SCORE_EMIT  1   /* sweep 2 of the scoring: per-token sums                    */
-#define DKV_STEP_POOL        2   /* unused: pooling is fused into sweep 2 */
-#define DKV_STEP_SELECT      3
-#define DKV_STEP_GATHER      4
-#define DKV_STEP_REBUDGET    5
-#define DKV_STEP_SHRINK      6
+#define DKV_STEP_SCORE_EMIT  1   /* sweep 2 of the scoring: per-token sums, pooled             */
+#define DKV_STEP_SELECT      2
+#define DKV_STEP_GATHER      3
+#define DKV_STEP_REBUDGET    4
+#define DKV_STEP_SHRINK      5
 #define DKV_N_STEPS          8
 int dkv_profile(dkv_ctx* ctx, int enable);
 int dkv_profile_read(dkv_ctx* ctx, double* ms, int64_t* launches);

@@ -16,7 +16,8 @@ LIB_PATH = os.path.join(HERE, "libdkv.so")
 EXPORTS = [
     "dkv_create", "dkv_destroy", "dkv_reset", "dkv_score", "dkv_score_static", "dkv_score_lse", "dkv_set_scores", "dkv_select_topk", "dkv_rebudget",
     "dkv_compact", "dkv_compact_all", "dkv_run_prefill_pass", "dkv_run_prefill_pass_host", "dkv_get_counts",
-    "dkv_layer_views", "dkv_kept_sorted", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status", "dkv_profile", "dkv_profile_read", "dkv_launch_count", "dkv_last_cuda_error",
+    "dkv_layer_views", "dkv_kept_sorted", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status",
+    "dkv_static_last_status", "dkv_set_wait_limit", "dkv_debug_withhold_tile", "dkv_profile", "dkv_profile_read", "dkv_launch_count", "dkv_last_cuda_error",
     "dkv_strerror", "dkv_version",
 ]
 
@@ -69,6 +70,9 @@ def load() -> ctypes.CDLL:
         "dkv_budget_views": [vp, pp, pp, pp, pp],
         "dkv_memcpy_to_host": [vp, vp, vp, ctypes.c_uint64, vp],
         "dkv_last_status": [vp, vp],
+        "dkv_static_last_status": [vp],
+        "dkv_set_wait_limit": [vp, ctypes.c_int64],
+        "dkv_debug_withhold_tile": [vp, i32, i32],
         "dkv_profile": [vp, ctypes.c_int],
         "dkv_profile_read": [vp, vp, vp],
         "dkv_last_cuda_error": [vp],
@@ -248,7 +252,21 @@ def dkv_last_status(ctx: int):
     return code, list(buf)
 
 
-STEP_NAMES = ["score_stats", "score_emit", "pool", "select", "gather", "rebudget", "shrink", "other"]
+def dkv_static_last_status():
+    buf = (ctypes.c_int32 * 8)()
+    code = load().dkv_static_last_status(buf)
+    return code, list(buf)
+
+
+def dkv_set_wait_limit(ctx: int, clock_ticks: int) -> None:
+    _check(load().dkv_set_wait_limit(ctx, clock_ticks), "dkv_set_wait_limit")
+
+
+def dkv_debug_withhold_tile(ctx: int, sweep: int, tile: int) -> None:
+    _check(load().dkv_debug_withhold_tile(ctx, sweep, tile), "dkv_debug_withhold_tile")
+
+
+STEP_NAMES = ["score_stats", "score_emit", "select", "gather", "rebudget", "shrink", "other6", "other7"]
 
 
 def dkv_profile(ctx: int, enable: bool) -> None:

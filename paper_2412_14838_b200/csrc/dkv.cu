@@ -20,6 +20,7 @@ using namespace dkv;
 struct ProfRec { cudaEvent_t a, b; int step; int launches; };
 
 constexpr int kSideStreams = 4;
+constexpr int kSelMaxSmem = DKV_MAX_LAYER_BUDGET * 8 + DKV_MAX_LAYER_BUDGET * 4;
 
 struct dkv_ctx {
   dkv_config cfg;
@@ -47,6 +48,9 @@ struct dkv_ctx {
   int n_sms, tc_grid, tc_slots;
   int pass_taper;       // group sizes halve towards the end of the pass
   int pass_group;       // layers per scoring launch of dkv_run_prefill_pass (1..tc::kMaxGroup)
+  bool emit_backward;   // sweep 2 walks every CTA's slice from the end to the start
+  long long wait_cycles;   // limit of the scoring kernel's mbarrier waits (dkv_set_wait_limit)
+  int withhold_sweep, withhold_tile;   // test hook of dkv_debug_withhold_tile (-1: off)
   float2* d_tc_stats;   // [3][kMaxGroup*Bt*Hkv][tc_slots][256]: partial softmax statistics, three jobs in rotation
   cudaStream_t hi;      // scoring launches of dkv_run_prefill_pass: highest priority, so that a freed SM goes to a
                         // waiting scoring CTA before the side streams' many short CTAs
@@ -93,10 +97,12 @@ int cuda_fail(dkv_ctx* c, cudaError_t e) {
     cudaError_t e__ = (call);                                 \
     if (e__ != cudaSuccess) return cuda_fail((ctx), e__);     \
   } while (0)
+// After a launch: a launch error is reported once and cleared (cudaGetLastError), so that a refused launch
+// does not make every later call of every context fail.
 #define DKV_LAUNCHED(ctx)                                     \
   do {                                                        \
     (ctx)->launches++;                                        \
-    cudaError_t e__ = cudaPeekAtLastError();                  \
+    cudaError_t e__ = cudaGetLastError();                     \
     if (e__ != cudaSuccess) return cuda_fail((ctx), e__);     \
   } while (0)
 
@@ -138,6 +144,17 @@ int validate(const dkv_config* c) {
   if ((long long)c->window * (c->n_q_heads / c->n_kv_heads) > DKV_MAX_WINDOW_ROWS) return DKV_ERR_UNSUPPORTED;
   if ((long long)c->n_layers * c->batch * c->n_kv_heads * (long long)c->seq_len >= (1ll << 31)) return DKV_ERR_UNSUPPORTED;
   return DKV_OK;
+}
+
+// Measurement overrides from the environment, read once per context in dkv_create: an integer inside
+// [lo, hi], anything else (unset, not a number, out of range) gives the default.
+int env_int(const char* name, int dflt, int lo, int hi) {
+  const char* e = getenv(name);
+  if (!e || !*e) return dflt;
+  char* end = nullptr;
+  const long v = strtol(e, &end, 10);
+  if (end == e || *end != '\0' || v < lo || v > hi) return dflt;
+  return (int)v;
 }
 
 int check_layer(const dkv_ctx* c, int layer) {
@@ -190,13 +207,14 @@ bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, con
               int buf, tc::Maps* maps, tc::Params* p) {
   const Shape& s = c->s;
   const int heads = s.Bt * s.Hkv;
-  for (int i = 0; i < tc::kMaxGroup; ++i) {
-    const int j = i < nl ? i : 0;                          // unused entries repeat the first (never read)
-    if (!make_map(&maps->q[i], q[j], s.D, s.M, heads) || !make_map(&maps->k[i], k[j], s.D, s.S, heads)) return false;
-  }
+  memset(maps, 0, sizeof *maps);                           // entries past nl are never read
+  for (int i = 0; i < nl; ++i)
+    if (!make_map(&maps->q[i], q[i], s.D, s.M, heads) || !make_map(&maps->k[i], k[i], s.D, s.S, heads)) return false;
   p->S = s.S; p->P = s.P; p->ws = s.ws; p->M = s.M; p->D = s.D; p->heads = nl * heads; p->half = s.pool / 2;
-  p->nl = nl; p->hpl = heads; p->rev = 0;
-  p->back = (mode == tc::kEmit && !getenv("DKV_EMIT_FORWARD")) ? 1 : 0;
+  p->nl = nl; p->hpl = heads;
+  p->back = (mode == tc::kEmit && c->emit_backward) ? 1 : 0;
+  p->wait_cycles = c->wait_cycles;
+  p->withhold_tile = c->withhold_sweep == mode ? c->withhold_tile : -1;
   p->tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
   p->nq16 = (s.M + 15) / 16 * 16;
   p->nmblk = (s.M + 127) / 128;
@@ -223,11 +241,10 @@ int launch_score(dkv_ctx* c, int stats_layer, int sn, const void* const* sq, con
   tc::Maps m0, m1;
   tc::Params j0, j1;
   memset(&j0, 0, sizeof j0); memset(&j1, 0, sizeof j1);
+  memset(&m0, 0, sizeof m0); memset(&m1, 0, sizeof m1);
   j0.mode = j1.mode = tc::kNone;
   if (emit_layer >= 0 && !make_job(c, tc::kEmit, emit_layer, en, eq, ek, scores_out, ebuf, &m0, &j0)) return DKV_ERR_CUDA;
   if (stats_layer >= 0 && !make_job(c, tc::kStats, stats_layer, sn, sq, sk, nullptr, sbuf, &m1, &j1)) return DKV_ERR_CUDA;
-  if (emit_layer < 0) m0 = m1;
-  if (stats_layer < 0) m1 = m0;
   ProfScope ps(c, stats_layer >= 0 ? DKV_STEP_SCORE_STATS : DKV_STEP_SCORE_EMIT, 1, st);
   tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(m0, m1, j0, j1);
   DKV_LAUNCHED(c);
@@ -535,7 +552,7 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
     // leave some SMs to the select / gather / update kernels that dkv_run_prefill_pass runs beside the scoring:
     // with grouped launches up to four layers' selects (one CTA per head) are in flight at once
     int side = 4 * heads < c->n_sms * 2 / 9 ? 4 * heads : c->n_sms * 2 / 9;
-    if (const char* e = getenv("DKV_SIDE_SMS")) side = atoi(e);
+    side = env_int("DKV_SIDE_SMS", side, 0, c->n_sms - 1);
     int score_sms = c->n_sms - side;
     if (score_sms < 1) score_sms = 1;
     c->tc_grid = (int)(total_tiles < score_sms ? total_tiles : score_sms);
@@ -548,16 +565,12 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
       }
     c->tc_slots = slots;
     // layers per scoring launch of the pass: enough that a CTA's share of a job is some tens of tiles
-    c->pass_group = total_tiles / c->tc_grid < 8 ? tc::kMaxGroup : 4;
-    if (const char* e = getenv("DKV_PASS_GROUP")) c->pass_group = atoi(e);
-    if (c->pass_group < 1) c->pass_group = 1;
-    if (c->pass_group > tc::kMaxGroup) c->pass_group = tc::kMaxGroup;
-    c->n_side = kSideStreams;
-    c->pass_taper = 0;
-    if (const char* e = getenv("DKV_PASS_TAPER")) c->pass_taper = atoi(e);
-    if (const char* e = getenv("DKV_SIDE_STREAMS")) c->n_side = atoi(e);
-    if (c->n_side < 1) c->n_side = 1;
-    if (c->n_side > kSideStreams) c->n_side = kSideStreams;
+    c->pass_group = env_int("DKV_PASS_GROUP", total_tiles / c->tc_grid < 8 ? tc::kMaxGroup : 4, 1, tc::kMaxGroup);
+    c->pass_taper = env_int("DKV_PASS_TAPER", 0, 0, 1);
+    c->n_side = env_int("DKV_SIDE_STREAMS", kSideStreams, 1, kSideStreams);
+    c->emit_backward = env_int("DKV_EMIT_FORWARD", 0, 0, 1) == 0;
+    c->wait_cycles = tc::kDefaultWaitCycles;
+    c->withhold_sweep = c->withhold_tile = -1;
   }
   const size_t bl = (size_t)s.Bt * s.L;
 #define TRY(call) if (e == cudaSuccess) e = (call)
@@ -582,7 +595,7 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaEventCreateWithFlags(&c->ev_gjoin, cudaEventDisableTiming));
   c->pass_key = new (std::nothrow) std::vector<const void*>();
   if (!c->pass_key) { free_all(c); delete c; return DKV_ERR_NOMEM; }
-  c->use_graph = getenv("DKV_NO_GRAPH") == nullptr;
+  c->use_graph = env_int("DKV_NO_GRAPH", 0, 0, 1) == 0;
   TRY(cudaStreamCreateWithFlags(&c->upd, cudaStreamNonBlocking));
   {
     int least = 0, greatest = 0;
@@ -606,8 +619,10 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
     c->sel_reg = (s.P + kSelThreads - 1) / kSelThreads <= kRegChunk;
     c->sel_smem = (size_t)c->sort_n * 8 + (size_t)s.Blc * 4;
   }
-  TRY(cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem));
-  TRY(cudaFuncSetAttribute(select_topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem));
+  // The attribute belongs to the function, not to this context: always the most any valid configuration needs
+  // (sort keys 8 B and positions 4 B for DKV_MAX_LAYER_BUDGET entries), so that contexts do not undo each other.
+  TRY(cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelMaxSmem));
+  TRY(cudaFuncSetAttribute(select_topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelMaxSmem));
 #undef TRY
   if (e != cudaSuccess) {
     rc = e == cudaErrorMemoryAllocation ? DKV_ERR_NOMEM : DKV_ERR_CUDA;
@@ -885,15 +900,18 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   if (need > DKV_STATIC_SCRATCH_BYTES) return DKV_ERR_TOO_LARGE;
   cudaStream_t st = as_stream(stream);
   tc::Maps maps;
-  for (int i = 0; i < tc::kMaxGroup; ++i)
-    if (!make_map(&maps.q[i], q_win, D, M, heads) || !make_map(&maps.k[i], k, D, S, heads)) return DKV_ERR_CUDA;
+  memset(&maps, 0, sizeof maps);
+  if (!make_map(&maps.q[0], q_win, D, M, heads) || !make_map(&maps.k[0], k, D, S, heads)) return DKV_ERR_CUDA;
   if (cudaMemsetAsync(su.ptr, 0, 256, st) != cudaSuccess) return DKV_ERR_CUDA;   // status words start at zero
   tc::Params p, none;
   memset(&p, 0, sizeof p);
   memset(&none, 0, sizeof none);
   none.mode = tc::kNone;
   p.S = S; p.P = P; p.ws = cfg->window; p.M = M; p.D = D; p.heads = heads; p.half = cfg->pool_kernel / 2;
-  p.nl = 1; p.hpl = heads; p.rev = 0;
+  p.nl = 1; p.hpl = heads;
+  p.back = 0;
+  p.wait_cycles = tc::kDefaultWaitCycles;
+  p.withhold_tile = -1;
   p.tph = tph; p.nq16 = (M + 15) / 16 * 16; p.nmblk = (M + 127) / 128;
   p.slots = slots; p.m_stride = 256;
   p.scale2 = kLog2e / sqrtf((float)D);
@@ -906,11 +924,11 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   p.mode = tc::kStats;
   p.idesc = make_idesc(128, 128);
   tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(maps, maps, p, none);
-  if (cudaPeekAtLastError() != cudaSuccess) return DKV_ERR_CUDA;
+  if (cudaGetLastError() != cudaSuccess) return DKV_ERR_CUDA;
   p.mode = tc::kEmit;
   p.idesc = make_idesc(128, p.nq16);
   tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(maps, maps, none, p);
-  if (cudaPeekAtLastError() != cudaSuccess) return DKV_ERR_CUDA;
+  if (cudaGetLastError() != cudaSuccess) return DKV_ERR_CUDA;
   return DKV_OK;
 }
 
@@ -925,8 +943,32 @@ int dkv_last_status(dkv_ctx* c, int32_t* host_status) {
   if (!c || !host_status) return DKV_ERR_INVALID_ARG;
   DKV_CUDA(c, cudaDeviceSynchronize());
   DKV_CUDA(c, cudaMemcpy(host_status, c->d_status, sizeof(int) * 8, cudaMemcpyDeviceToHost));
+  if (host_status[0] != 0) DKV_CUDA(c, cudaMemset(c->d_status, 0, sizeof(int) * 8));   // reported once
   host_status[1] = (int32_t)(c->launches & 0x7FFFFFFF);
-  return host_status[0] == 0 ? DKV_OK : host_status[0];
+  return host_status[0] == 0 ? DKV_OK : DKV_ERR_TIMEOUT;
+}
+
+int dkv_static_last_status(int32_t* host_status) {
+  if (!host_status) return DKV_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return DKV_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(host_status, g_static_scratch, sizeof(int) * 8) != cudaSuccess) return DKV_ERR_CUDA;
+  host_status[1] = 0;
+  return host_status[0] == 0 ? DKV_OK : DKV_ERR_TIMEOUT;
+}
+
+int dkv_set_wait_limit(dkv_ctx* c, int64_t clock_ticks) {
+  if (!c || clock_ticks < 1000) return DKV_ERR_INVALID_ARG;
+  c->wait_cycles = clock_ticks;
+  if (c->pass_exec) { cudaGraphExecDestroy(c->pass_exec); c->pass_exec = nullptr; }   // recorded with the old limit
+  return DKV_OK;
+}
+
+int dkv_debug_withhold_tile(dkv_ctx* c, int32_t sweep, int32_t tile) {
+  if (!c || (tile >= 0 && sweep != 1 && sweep != 2)) return DKV_ERR_INVALID_ARG;
+  c->withhold_sweep = tile >= 0 ? sweep : -1;
+  c->withhold_tile = tile >= 0 ? tile : -1;
+  if (c->pass_exec) { cudaGraphExecDestroy(c->pass_exec); c->pass_exec = nullptr; }
+  return DKV_OK;
 }
 
 int dkv_profile(dkv_ctx* c, int enable) {

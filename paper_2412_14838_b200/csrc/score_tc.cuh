@@ -37,7 +37,8 @@ constexpr int kKRegion = kStages * 2 * kHalfBytes;    // ring of 128 x 128 tiles
 constexpr int kMiscBytes = 1024 /*lse*/ + 3 * 256 * 8 /*merge*/;
 constexpr int kRawBytes = 2 * kMaxSegTiles * kTileKeys * 4;   // sweep 2: one partial-sum array per column half
 constexpr int kSmemBytes = 1024 /*align*/ + kQRegion + kKRegion + kMiscBytes + kRawBytes + 256 /*barriers*/;
-constexpr long long kWaitCycles = 4000000000ll;       // ~2 s: a wait that long is reported, not spun on
+constexpr long long kDefaultWaitCycles = 4000000000ll;  // ~2 s: a wait that long is reported, not spun on
+constexpr long long kDrainCycles = 2000000ll;           // ~1 ms: wait for own copies / MMAs in flight after an abort
 
 enum Mode { kNone = 0, kStats = 1, kEmit = 2 };
 
@@ -61,20 +62,17 @@ struct Params {
   const float* lse_in;     // sweep 2: caller's natural-log normalisers [heads][M] (then sweep 1 never ran), or null
   int nl;                  // layers this job covers (1..kMaxGroup); `heads` counts the heads of all of them
   int hpl;                 // heads per layer
-  int rev;                 // 1: the job walks its layers from the last to the first
   int back;                // sweep 2: 1 = every CTA walks its slice from the end to the start, so that it begins
                            // with the keys sweep 1 streamed last (those still in L2)
+  long long wait_cycles;   // limit of every mbarrier wait, in clock64 ticks
+  int withhold_tile;       // test hook: CTA 0 never loads its key tile number `withhold_tile` of this job (-1: off),
+                           // so that the wait for it runs out and the timeout path can be exercised
 };
 
 constexpr int kMaxGroup = 8;               // layers one job may cover
 struct Maps {                              // tensor maps of a job's layers, in storage order
   CUtensorMap q[kMaxGroup], k[kMaxGroup];
 };
-
-// Head index in storage order (layer-major) of the head a job visits as number `bh`.
-__device__ __forceinline__ int stored_head(const Params& p, int bh) {
-  return p.rev ? (p.nl - 1 - bh / p.hpl) * p.hpl + bh % p.hpl : bh;
-}
 
 // ------------------------------------------------------------------------------------------ PTX
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -97,19 +95,28 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after kWaitCycles, records the failure and lets the kernel run to its end.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+// Bounded wait: gives up after `limit` clock ticks, records the failure (status[0] = the first wait site that
+// gave up, status[2] = its CTA) and lets the kernel run to its end: once the CTA's abort flag is up no wait
+// blocks, no further copy or MMA is issued, and the CTA drains what it has in flight before it frees its
+// tensor memory.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+                                          long long limit) {
   if (*abort_flag) return;
   if (mbar_try(bar, parity)) return;
   const long long t0 = clock64();
   while (!mbar_try(bar, parity)) {
     if (*abort_flag) return;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
-      atomicCAS(status, 0, code);
+      if (atomicCAS(status, 0, code) == 0) status[2] = (int)blockIdx.x;
       return;
     }
   }
+}
+// After an abort: wait a short while for something of this CTA's own that is still in flight.  Never records.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try(bar, parity)) if (clock64() - t0 > kDrainCycles) return;
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
   asm volatile(
@@ -247,7 +254,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
   float2* merge_s = reinterpret_cast<float2*>(lse_s + 256);            // [3][256] partials of column parts 1..3 (sweep 1)
   float* raw_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(lse_s) + kMiscBytes);   // [half][kMaxSegTiles * 128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(raw_s) + kRawBytes);
-  // barriers: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2], q_full
+  // barriers: full[kStages], empty[kStages], tmem_full[4], tmem_empty[4], q_full, drain[2]
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
   const uint32_t bar0 = smem_u32(bars);
@@ -256,6 +263,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
   auto TFULL = [&](int t) { return bar0 + 8u * (2 * kStages + t); };
   auto TEMPTY = [&](int t) { return bar0 + 8u * (2 * kStages + 4 + t); };
   const uint32_t QFULL = bar0 + 8u * (2 * kStages + 8);
+  auto DRAIN = [&](int i) { return bar0 + 8u * (2 * kStages + 9 + i); };   // one per MMA issuer, used after an abort only
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &abort_s;
@@ -265,6 +273,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
     for (int s = 0; s < kStages; ++s) { mbar_init(FULL(s), 1); mbar_init(EMPTY(s), 1); }
     for (int t = 0; t < 4; ++t) { mbar_init(TFULL(t), 1); mbar_init(TEMPTY(t), 8); }
     mbar_init(QFULL, 1);
+    mbar_init(DRAIN(0), 1); mbar_init(DRAIN(1), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -279,40 +288,54 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int tile = 0;
+      int tile = 0, nq = 0;
+      int last_on[kStages];                    // last tile whose copy went to each ring stage (-1: none)
+      for (int s = 0; s < kStages; ++s) last_on[s] = -1;
       for (int jb = 0; jb < 2; ++jb) {
         const Params& p = jb ? job1 : job0;
         if (p.mode == kNone) continue;
         const Maps& maps = jb ? maps1 : maps0;
         const int halves = p.D / 64;
         const uint32_t tile_bytes = (uint32_t)halves * kHalfBytes;
+        const int withhold = blockIdx.x == 0 ? p.withhold_tile : -1;
         SegIter it(p, blockIdx.x, gridDim.x);
         Seg sg;
+        int job_tile = 0;
         while (it.next(sg)) {
-          const int nb = stored_head(p, sg.bh), hh = nb % p.hpl;
-          const CUtensorMap* q_map = &maps.q[nb / p.hpl];
-          const CUtensorMap* k_map = &maps.k[nb / p.hpl];
+          const int hh = sg.bh % p.hpl;
+          const CUtensorMap* q_map = &maps.q[sg.bh / p.hpl];
+          const CUtensorMap* k_map = &maps.k[sg.bh / p.hpl];
           if (sg.new_head) {
             // every MMA that read the previous queries must have finished: the last tile of either issuer
             for (int last = tile - 1; last >= 0 && last >= tile - 2; --last)
-              mbar_wait(EMPTY(last % kStages), (last / kStages) & 1, abort_flag, p.status, 101);
+              mbar_wait(EMPTY(last % kStages), (last / kStages) & 1, abort_flag, p.status, 101, p.wait_cycles);
             if (!*abort_flag) {
               mbar_expect_tx(QFULL, (uint32_t)(p.nmblk * halves) * kHalfBytes);
               for (int h = 0; h < halves; ++h)
                 for (int mb = 0; mb < p.nmblk; ++mb)
                   tma_load_3d(smem_u32(q_smem + h * (2 * kHalfBytes) + mb * kHalfBytes), q_map, QFULL, 64 * h, 128 * mb, hh);
+              ++nq;
             }
           }
-          for (int i = 0; i < sg.ntiles; ++i, ++tile) {
+          for (int i = 0; i < sg.ntiles; ++i, ++tile, ++job_tile) {
             const int s = tile % kStages, n = tile / kStages;
-            mbar_wait(EMPTY(s), (n & 1) ^ 1, abort_flag, p.status, 102);
+            mbar_wait(EMPTY(s), (n & 1) ^ 1, abort_flag, p.status, 102, p.wait_cycles);
             if (*abort_flag) break;
+            if (job_tile == withhold) continue;          // test hook: this tile never arrives
             mbar_expect_tx(FULL(s), tile_bytes);
             for (int h = 0; h < halves; ++h)
               tma_load_3d(smem_u32(k_smem + (s * 2 + h) * kHalfBytes), k_map, FULL(s), 64 * h, sg.key0 + i * kTileKeys, hh);
+            last_on[s] = tile;
           }
           if (*abort_flag) break;
         }
+        if (*abort_flag) break;
+      }
+      if (*abort_flag) {
+        // copies of this CTA that may still be on their way must land before its shared memory is given up
+        for (int s = 0; s < kStages; ++s)
+          if (last_on[s] >= 0) mbar_drain(FULL(s), (last_on[s] / kStages) & 1);
+        if (nq > 0) mbar_drain(QFULL, (nq - 1) & 1);
       }
     }
   } else if (warp == 1 || warp == kMmaWarp2) {
@@ -338,11 +361,12 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
             if ((tile & 1) != which) continue;
             if (q_wait) {
               q_wait = false;
-              mbar_wait(QFULL, (nq - 1) & 1, abort_flag, p.status, 103);
+              mbar_wait(QFULL, (nq - 1) & 1, abort_flag, p.status, 103, p.wait_cycles);
             }
             const int s = tile % kStages, n = tile / kStages, t = tile & tmask, nt = tile >> tshift;
-            mbar_wait(FULL(s), n & 1, abort_flag, p.status, 104);
-            mbar_wait(TEMPTY(t), (nt & 1) ^ 1, abort_flag, p.status, 105);
+            mbar_wait(FULL(s), n & 1, abort_flag, p.status, 104, p.wait_cycles);
+            mbar_wait(TEMPTY(t), (nt & 1) ^ 1, abort_flag, p.status, 105, p.wait_cycles);
+            if (*abort_flag) continue;                   // nothing more is issued once a wait has run out
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(t * scols);
             if (p.mode == kStats) {
@@ -363,6 +387,11 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
             tc_commit(TFULL(t));      // the accumulator is complete
           }
         }
+      }
+      if (*abort_flag) {
+        // the MMAs this thread has issued must have finished before the tensor memory is freed
+        tc_commit(DRAIN(which));
+        mbar_drain(DRAIN(which), 0);
       }
     }
   } else {
@@ -388,7 +417,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
             if ((tile & 1) != grp) continue;                   // the other group's tile
             const int t = tile & tmask, nt = tile >> tshift;
-            mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 106);
+            mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 106, p.wait_cycles);
             tc_fence_after();
             const uint32_t taddr = lane_addr + (uint32_t)(t * scols + half * 64);
             const int kb0 = sg.key0 + i * kTileKeys + half * 64;
@@ -461,7 +490,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
           asm volatile("bar.sync 1, 512;" ::: "memory");
         } else {
           // ------------------------------------------------------------ sweep 2: one thread per key
-          const int nb = stored_head(p, sg.bh);              // sweep 1 filed its statistics in storage order
+          const int nb = sg.bh;
           if (sg.new_head && sid < 256) {
             // lse2 of every window row from the partial statistics of sweep 1
             const long long total = (long long)p.heads * p.tph;
@@ -488,7 +517,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
             if ((tile & 1) != grp) continue;                   // the other group's tile
             const int t = tile & tmask, nt = tile >> tshift;
-            mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 107);
+            mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 107, p.wait_cycles);
             tc_fence_after();
             const uint32_t taddr = lane_addr + (uint32_t)(t * scols);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;

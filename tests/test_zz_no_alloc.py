@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import dynamickv as O
 from paper_2412_14838_b200 import binding as B
 from paper_2412_14838_b200 import build, synth
 from tests import _util as U
@@ -38,12 +39,20 @@ def test_static_scoring_matches_the_context_path_twice_in_a_row():
                 want = torch.empty((w.Bt, w.Hkv, w.P), dtype=torch.float32, device="cuda")
                 got = torch.full_like(want, -1.0)
                 B.dkv_score(ctx, layer, q, k, want)
+                torch.cuda.synchronize()
+                free_before = torch.cuda.mem_get_info()[0]
                 B.dkv_score_static(B.config_of(w), q, k, got)
                 torch.cuda.synchronize()
+                if layer == 1:                           # past the first call's one-time set-up
+                    assert torch.cuda.mem_get_info()[0] == free_before, "the call took device memory"
+                code, status = B.dkv_static_last_status()
+                assert code == B.DKV_OK and status[0] == 0
                 want, got = want.cpu().numpy(), got.cpu().numpy()
                 assert (got >= 0).all(), "some scores were never written"
                 rel = np.abs(got - want) / np.maximum(want, U.TINY)
                 assert rel.max() <= U.REL_TOL, f"{w.name} call {layer}: off by {rel.max():.2e}"
+                ref = O.window_scores(synth.bf16_bits_to_f64(t["q"]), synth.bf16_bits_to_f64(t["k"]), w.ws, w.pool)
+                U.assert_scores_close(got, ref["score"], f"{w.name} call {layer} against the oracle")
         finally:
             B.dkv_destroy(ctx)
 
