@@ -16,7 +16,11 @@ prefix tokens, ``N = wt - ws``, ``B^l`` = ``Bl`` per-layer maximum, ``m`` update
 * ``budget_from_counts``   Eq. 5-6 with the ``int()`` truncations of Update_Buffer_Length.
 * ``rebudget``             Update_Buffer_Length as a whole + the "buffers only shrink" clamp.
 * ``shrink_rows``          Algorithm 1's truncation of every preceding layer's buffer.
-* ``run_prefill_pass``     Algorithm 1's loop over layers.
+* ``run_prefill_pass``     Algorithm 1's loop over layers (optionally scored from given log-denominators).
+* ``decode_attention``     Eq. 1 applied to one new query over a layer's compressed, ragged cache (Section 4.3:
+                           decoding runs unchanged over whatever the prefill phase kept).
+* ``policy_counts``, ``positions_sinks_recent``   the fixed-pattern budgets the paper compares with (the
+                           "Baselines" paragraph of Section 5.1), as budget / position policies only.
 
 Alternative readings, off by default, selectable per call: the window MEAN instead of the sum, an
 average pool (``avg_pool_same``), the pro-rata budget ``B = N * l`` at an intermediate update, and
@@ -31,6 +35,10 @@ of odd width over the prefix, borders ignoring the missing neighbours; ties are 
 lowest index (flat index, layer-major, for the global top-K); ``Norm`` is a positive scaling,
 so Eq. 5 is evaluated in exact integers; counts never grow.
 
+For the decode step: a hand-worked 3-key case (tests/golden/decode_handworked.txt), torch's masked softmax
+attention on the padded buffers, invariance under a permutation of the kept rows, the single-row and
+equal-keys special cases.  For the policies: hand-worked schedules (tests/golden/policies_handworked.txt),
+their sums and monotonicity.
 Pins (tests/test_oracle_*.py): closed forms for zero keys, probability-mass conservation,
 a hand-worked 3-key softmax, an independent torch softmax / max_pool1d route, torch's logsumexp and the
 ln 6 of the hand-worked case for the log-denominators, permutation
@@ -276,14 +284,16 @@ def shrink_rows(buf: np.ndarray, idx: np.ndarray, rank: np.ndarray, valid: int, 
 
 
 def run_prefill_pass(layer_fn, L: int, *, ws: int, pool: int, N: int, Bl: int, m: int, pool_kind: int = 0,
-                     window_mean: bool = False, prorata: bool = False, minmax: bool = False) -> Dict[str, object]:
+                     window_mean: bool = False, prorata: bool = False, minmax: bool = False,
+                     lse_fn=None) -> Dict[str, object]:
     """Algorithm 1's loop over the layers, for all samples.
 
     ``layer_fn(l)`` returns one layer's inputs as a dict: ``q`` [Bt,Hq,ws,D] and ``k`` [Bt,Hkv,S,D]
     in float64 (used for scoring), and ``k_rows`` / ``v_rows`` [Bt,Hkv,S,D] in any dtype (the
     rows that are moved; typically the raw bf16 bit patterns).  A layer's full K/V is only
     touched while that layer is processed, as in the paper's prefill loop.  If ``L % m != 0``
-    one more update runs after the last layer.
+    one more update runs after the last layer.  With ``lse_fn`` given, ``lse_fn(l)`` supplies layer ``l``'s
+    log-denominators [Bt,Hq,ws] and the scores come from ``window_scores_from_lse`` (one sweep).
 
     Returns per layer: ``score`` [Bt,Hkv,P]; ``idx``/``rank`` lists [L][Bt][Hkv] of the final kept
     positions and their ranks; ``kb``/``vb`` lists [L][Bt][Hkv] of final buffers (kept rows then
@@ -318,7 +328,11 @@ def run_prefill_pass(layer_fn, L: int, *, ws: int, pool: int, N: int, Bl: int, m
         P = S - ws
         if counts is None:
             counts = np.zeros((Bt, L), dtype=np.int64)
-        sc = window_scores(inp["q"], inp["k"], ws, pool, pool_kind=pool_kind, window_mean=window_mean)["score"]
+        if lse_fn is None:
+            sc = window_scores(inp["q"], inp["k"], ws, pool, pool_kind=pool_kind, window_mean=window_mean)["score"]
+        else:
+            sc = window_scores_from_lse(inp["q"], inp["k"], lse_fn(l), ws, pool, pool_kind=pool_kind,
+                                        window_mean=window_mean)["score"]
         scores.append(sc)
         for lst in (idx, rank, kb, vb, first_idx, first_rank):
             lst.append([[None] * Hkv for _ in range(Bt)])
@@ -337,3 +351,57 @@ def run_prefill_pass(layer_fn, L: int, *, ws: int, pool: int, N: int, Bl: int, m
         update(L)
     return {"score": scores, "idx": idx, "rank": rank, "kb": kb, "vb": vb, "counts": counts,
             "first_idx": first_idx, "first_rank": first_rank, "updates": updates}
+
+
+# --------------------------------------------------------------------------- decoding over the compressed cache
+def decode_attention(q_dec: np.ndarray, kb, vb, lengths: Sequence[int]) -> np.ndarray:
+    """Eq. 1 for newly generated tokens over one layer's compressed cache (Section 4.3: the decoding phase
+    is the model's own attention, run over what the prefill phase kept).
+
+    ``q_dec`` [Bt, Hq, nq, D] float64: ``nq`` independent queries per sample and query head.  ``kb`` and
+    ``vb`` are indexable as ``[b][h]`` and give that KV head's buffer [rows, D] (kept prefix rows followed by
+    the ``ws`` window rows; rows past ``lengths[b]`` are padding and never read).  Query head ``hq`` reads KV
+    head ``hq // G``.  Every query sees all ``lengths[b]`` rows: the cache holds only earlier positions.
+    Returns [Bt, Hq, nq, D]: ``softmax(q K^T / sqrt(d_k)) V`` row by row.
+    """
+    Bt, Hq, nq, D = q_dec.shape
+    Hkv = len(kb[0])
+    assert Hq % Hkv == 0
+    G = Hq // Hkv
+    out = np.zeros((Bt, Hq, nq, D), dtype=np.float64)
+    for b in range(Bt):
+        n = int(lengths[b])
+        for hq in range(Hq):
+            K = np.asarray(kb[b][hq // G], dtype=np.float64)[:n]
+            V = np.asarray(vb[b][hq // G], dtype=np.float64)[:n]
+            for i in range(nq):
+                logits = (K @ q_dec[b, hq, i]) / np.sqrt(np.float64(D))
+                e = np.exp(logits - logits.max())
+                out[b, hq, i] = (e / e.sum()) @ V
+    return out
+
+
+# --------------------------------------------------------------------------- fixed-pattern policies
+def policy_counts(policy: str, L: int, N: int) -> List[int]:
+    """Per-layer budgets of the fixed-pattern methods the paper compares with, as plain schedules (no
+    scores involved): ``"uniform"`` keeps the same ``N`` tokens per head in every layer (the fixed
+    per-layer cache of SnapKV-like methods); ``"pyramid"`` decreases monotonically with depth (the pyramid
+    pattern): ``N + floor(N * (L - 1 - 2 i) / (2 (L - 1)))`` for layer ``i``, i.e. linearly from about
+    ``3N/2`` at the first layer to ``N/2`` at the last, summing to ``N * L`` up to the floors (``N``
+    when ``L = 1``).  The kept tokens are then the best ``count_i`` of each head under Eq. 3's order."""
+    if policy == "uniform":
+        return [int(N)] * L
+    if policy == "pyramid":
+        if L == 1:
+            return [int(N)]
+        return [int(N) + (int(N) * (L - 1 - 2 * i)) // (2 * (L - 1)) for i in range(L)]
+    raise ValueError(f"unknown policy {policy!r}")
+
+
+def positions_sinks_recent(P: int, n_sink: int, n_recent: int) -> np.ndarray:
+    """Kept prefix positions of a sinks-plus-recent cache (attention sinks and a rolling window of the most
+    recent tokens, StreamingLLM-like): the first ``n_sink`` and the last ``n_recent`` of the ``P`` prefix
+    positions, ascending, each once (the two ranges merge when they meet)."""
+    n_sink, n_recent = max(0, min(int(n_sink), P)), max(0, min(int(n_recent), P))
+    first_recent = max(P - n_recent, n_sink)
+    return np.concatenate([np.arange(n_sink), np.arange(first_recent, P)]).astype(np.int64)

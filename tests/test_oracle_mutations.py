@@ -47,6 +47,22 @@ def _checks(o):
     out.append(("shrink_only", res["counts"] == [3, 0]))
     # global ties to the lower layer
     out.append(("global_ties", o.global_topk_counts([np.full((1, 4), 0.5)] * 2, 4).tolist() == [4, 0]))
+    # decode step: the hand-worked 3-key case (d_k = 4, probabilities 1/6, 2/6, 3/6), padding never read
+    qd = np.zeros((1, 4, 1, 4)); qd[0, :, 0, 0] = 2.0               # four query heads on two KV heads
+    kd = np.zeros((2, 5, 4)); vd = np.zeros((2, 5, 4))
+    for j in range(3):
+        kd[:, j, 0] = math.log(j + 1.0)
+        vd[0, j] = [6.0 * (j + 1), 1.0, -(j + 1.0), 0.0]
+        vd[1, j] = [1.0, 0.0, 0.0, 0.0]
+    kd[:, 3:] = 50.0; vd[:, 3:] = 1e6
+    got = o.decode_attention(qd, [kd], [vd], [3])
+    out.append(("decode", np.allclose(got[0, 0, 0], [14.0, 1.0, -7.0 / 3.0, 0.0], rtol=1e-12, atol=1e-12)
+                and np.allclose(got[0, 1, 0], [14.0, 1.0, -7.0 / 3.0, 0.0], rtol=1e-12, atol=1e-12)
+                and np.allclose(got[0, 2, 0], [1.0, 0.0, 0.0, 0.0], atol=1e-12)
+                and np.allclose(got[0, 3, 0], [1.0, 0.0, 0.0, 0.0], atol=1e-12)))
+    # policies: floors towards minus infinity, first positions then the most recent
+    out.append(("pyramid", o.policy_counts("pyramid", 5, 10) == [15, 12, 10, 7, 5]))
+    out.append(("sinks", o.positions_sinks_recent(10, 2, 3).tolist() == [0, 1, 7, 8, 9]))
     return out
 
 
@@ -116,7 +132,36 @@ def _global_high_layer(history, k):
     return O.global_topk_counts(list(history)[::-1], k)[::-1]
 
 
+def _decode_no_scale(q_dec, kb, vb, lengths):
+    return O.decode_attention(q_dec * math.sqrt(q_dec.shape[-1]), kb, vb, lengths)
+
+
+def _decode_wrong_group(q_dec, kb, vb, lengths):                       # query head hq reads KV head hq % Hkv
+    Hkv = len(kb[0])
+    perm = [(hq % Hkv) * (q_dec.shape[1] // Hkv) + hq // Hkv for hq in range(q_dec.shape[1])]
+    return O.decode_attention(q_dec, kb, vb, lengths)[:, perm]
+
+
+def _decode_reads_padding(q_dec, kb, vb, lengths):
+    return O.decode_attention(q_dec, kb, vb, [int(n) + 1 for n in lengths])
+
+
+def _pyramid_truncating(policy, L, N):
+    if policy != "pyramid" or L == 1:
+        return O.policy_counts(policy, L, N)
+    return [N + int(N * (L - 1 - 2 * i) / (2 * (L - 1))) for i in range(L)]      # rounds towards zero
+
+
+def _sinks_from_the_end(P, n_sink, n_recent):
+    return O.positions_sinks_recent(P, n_recent, n_sink)
+
+
 MUTANTS = {
+    "decode: no 1/sqrt(d_k)": dict(decode_attention=_decode_no_scale),
+    "decode: wrong KV head for a query head": dict(decode_attention=_decode_wrong_group),
+    "decode: one padding row read": dict(decode_attention=_decode_reads_padding),
+    "pyramid: truncation instead of floor": dict(policy_counts=_pyramid_truncating),
+    "sinks and recents swapped": dict(positions_sinks_recent=_sinks_from_the_end),
     "no 1/sqrt(d_k)": dict(softmax_rows_causal=_softmax_no_scale),
     "mean over window rows": dict(reduce_rows=lambda A: A.mean(axis=0)),
     "no causal mask in the window": dict(softmax_rows_causal=_softmax_no_causal),
