@@ -188,12 +188,53 @@ int dkv_compact_all(dkv_ctx* ctx, int32_t upto_layer, void* const* kb, void* con
 int dkv_run_prefill_pass(dkv_ctx* ctx, const void* const* q_win, const void* const* k, const void* const* v,
                          void* const* kb, void* const* vb, void* stream);
 
+/* Algorithm 1's loop when the caller's prefill attention kernel has already produced, for every layer, the
+ * log-denominators of the window rows (see dkv_score_lse): every layer is scored in one sweep over its keys.
+ * lse : HOST array of L device pointers, each fp32 [Bt, Hq, ws] (natural logarithm), 4-byte aligned.
+ * Everything else as dkv_run_prefill_pass, including the recording of the pass as a CUDA graph.  (Section 4.3
+ * notes that the scoring needs the window rows' attention probabilities explicitly, which a fused attention
+ * kernel does not return; its log-denominators are what it does return.) */
+int dkv_run_prefill_pass_lse(dkv_ctx* ctx, const void* const* q_win, const void* const* k, const void* const* v,
+                             const float* const* lse, void* const* kb, void* const* vb, void* stream);
+
 /* The same pass with all tensors in HOST memory (pinned memory recommended): each layer's q, k, v
  * are copied to device staging buffers owned by the context, processed, and after the last update
  * every layer's kb/vb (full fixed-stride buffers) and the counts are copied back.  Synchronises.
  * q_win, k, v, kb, vb : host arrays of L HOST pointers; counts_out : host int32 [Bt, L]. */
 int dkv_run_prefill_pass_host(dkv_ctx* ctx, const void* const* q_win, const void* const* k,
                               const void* const* v, void* const* kb, void* const* vb, int32_t* counts_out);
+
+/* Fixed-pattern budgets: the per-layer schedules of the methods the paper compares with (Section 5.1,
+ * "Baselines"), applied through the same select / compact kernels in place of Eq. 4-6.  Needs every layer
+ * selected.  count[b][i] = min(count[b][i], schedule_i) on the device; follow with dkv_compact_all (layers
+ * gathered later pick the new count up by themselves).
+ *   DKV_POLICY_UNIFORM : schedule_i = N in every layer (a fixed per-layer cache, as SnapKV-like methods keep).
+ *   DKV_POLICY_PYRAMID : schedule_i = N + floor(N (L-1-2i) / (2 (L-1))), falling linearly with depth from about
+ *                        3N/2 to N/2 (the pyramid pattern), summing to N*L up to the floors; N when L = 1.
+ *   counts_out : int32 [Bt, L] device copy of the counts after the call (optional). */
+#define DKV_POLICY_UNIFORM 0
+#define DKV_POLICY_PYRAMID 1
+int dkv_apply_policy(dkv_ctx* ctx, int32_t policy, int32_t* counts_out, void* stream);
+/* Selection by position, without scores, in place of dkv_select_topk for one layer: every head keeps the first
+ * n_sink and the last n_recent of its P prefix positions (attention sinks plus a window of the most recent
+ * tokens, as StreamingLLM-like methods keep), ascending, each once if the two ranges meet.  The kept number must
+ * not exceed Bl'.  Sets count[b][layer]; dkv_compact then gathers those rows.  Such a layer has no place in the
+ * global top-K: dkv_rebudget over it returns DKV_ERR_STATE. */
+int dkv_select_positions(dkv_ctx* ctx, int32_t layer, int32_t n_sink, int32_t n_recent, void* stream);
+
+/* Decoding over the compressed cache (Section 4.3: decoding is the model's own attention, Eq. 1, over what
+ * the prefill phase kept).  For layers [layer0, layer0 + n_layers), every sample b, query head hq and each of
+ * the nq new queries:  out = softmax(q . Kb^T / sqrt(D)) Vb  over the rows [0, count[b][layer] + ws) of KV head
+ * hq / G's buffers, the lengths being read from the context's device-side counts (they differ per layer).
+ * The nq queries of a sample are independent: each sees the whole compressed cache.
+ *   q_dec : HOST array of n_layers device pointers, bf16 [Bt, Hq, nq, D];  nq >= 1, G * nq <= 64
+ *   kb, vb: HOST arrays of n_layers device pointers, the buffers dkv_compact wrote (layers must be gathered)
+ *   out   : HOST array of n_layers device pointers, fp32 [Bt, Hq, nq, D]
+ * bf16 inputs, fp32 accumulation.  One launch covers up to 64 layers; partial results of the thread blocks
+ * that share a head go through a scratch array the context allocates on first use (and enlarges when a call
+ * needs more; that one call synchronises the device). */
+int dkv_decode_attend(dkv_ctx* ctx, int32_t layer0, int32_t n_layers, int32_t nq, const void* const* q_dec,
+                      const void* const* kb, const void* const* vb, float* const* out, void* stream);
 
 /* Copy the current counts to host int32 [Bt, L] (synchronises `stream`). */
 int dkv_get_counts(dkv_ctx* ctx, int32_t* host_counts, void* stream);
@@ -243,6 +284,7 @@ int dkv_debug_withhold_tile(dkv_ctx* ctx, int32_t sweep, int32_t tile);
 #define DKV_STEP_GATHER      3
 #define DKV_STEP_REBUDGET    4
 #define DKV_STEP_SHRINK      5
+#define DKV_STEP_DECODE      6
 #define DKV_N_STEPS          8
 int dkv_profile(dkv_ctx* ctx, int enable);
 int dkv_profile_read(dkv_ctx* ctx, double* ms, int64_t* launches);

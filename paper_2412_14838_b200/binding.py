@@ -15,7 +15,8 @@ LIB_PATH = os.path.join(HERE, "libdkv.so")
 
 EXPORTS = [
     "dkv_create", "dkv_destroy", "dkv_reset", "dkv_score", "dkv_score_static", "dkv_score_lse", "dkv_set_scores", "dkv_select_topk", "dkv_rebudget",
-    "dkv_compact", "dkv_compact_all", "dkv_run_prefill_pass", "dkv_run_prefill_pass_host", "dkv_get_counts",
+    "dkv_compact", "dkv_compact_all", "dkv_run_prefill_pass", "dkv_run_prefill_pass_lse", "dkv_run_prefill_pass_host",
+    "dkv_apply_policy", "dkv_select_positions", "dkv_decode_attend", "dkv_get_counts",
     "dkv_layer_views", "dkv_kept_sorted", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status",
     "dkv_static_last_status", "dkv_set_wait_limit", "dkv_debug_withhold_tile", "dkv_profile", "dkv_profile_read", "dkv_launch_count", "dkv_last_cuda_error",
     "dkv_strerror", "dkv_version",
@@ -64,6 +65,10 @@ def load() -> ctypes.CDLL:
         "dkv_compact_all": [vp, i32, pp, pp, vp],
         "dkv_run_prefill_pass": [vp, pp, pp, pp, pp, pp, vp],
         "dkv_run_prefill_pass_host": [vp, pp, pp, pp, pp, pp, vp],
+        "dkv_run_prefill_pass_lse": [vp, pp, pp, pp, pp, pp, pp, vp],
+        "dkv_apply_policy": [vp, i32, vp, vp],
+        "dkv_select_positions": [vp, i32, i32, i32, vp],
+        "dkv_decode_attend": [vp, i32, i32, i32, pp, pp, pp, pp, vp],
         "dkv_get_counts": [vp, vp, vp],
         "dkv_layer_views": [vp, i32, pp, pp],
         "dkv_kept_sorted": [vp, i32, vp, vp],
@@ -212,6 +217,31 @@ def dkv_run_prefill_pass_host(ctx: int, q_win: Sequence, k: Sequence, v: Sequenc
                                             _ptr_array(vb), _ptr(counts_out)), "dkv_run_prefill_pass_host")
 
 
+def dkv_run_prefill_pass_lse(ctx: int, q_win: Sequence, k: Sequence, v: Sequence, lse: Sequence, kb: Sequence,
+                             vb: Sequence, stream=None) -> None:
+    """The pass with every layer scored in one sweep from the window rows' log-denominators (see include/dkv.h)."""
+    _check(load().dkv_run_prefill_pass_lse(ctx, _ptr_array(q_win), _ptr_array(k), _ptr_array(v), _ptr_array(lse),
+                                           _ptr_array(kb), _ptr_array(vb), _stream(stream)), "dkv_run_prefill_pass_lse")
+
+
+DKV_POLICY_UNIFORM, DKV_POLICY_PYRAMID = 0, 1
+
+
+def dkv_apply_policy(ctx: int, policy: int, counts_out=None, stream=None) -> None:
+    _check(load().dkv_apply_policy(ctx, policy, _ptr(counts_out), _stream(stream)), "dkv_apply_policy")
+
+
+def dkv_select_positions(ctx: int, layer: int, n_sink: int, n_recent: int, stream=None) -> None:
+    _check(load().dkv_select_positions(ctx, layer, n_sink, n_recent, _stream(stream)), "dkv_select_positions")
+
+
+def dkv_decode_attend(ctx: int, layer0: int, n_layers: int, nq: int, q_dec: Sequence, kb: Sequence, vb: Sequence,
+                      out: Sequence, stream=None) -> None:
+    """Attention of nq new queries per sample over the compressed buffers of layers [layer0, layer0 + n_layers)."""
+    _check(load().dkv_decode_attend(ctx, layer0, n_layers, nq, _ptr_array(q_dec), _ptr_array(kb), _ptr_array(vb),
+                                    _ptr_array(out), _stream(stream)), "dkv_decode_attend")
+
+
 def dkv_get_counts(ctx: int, host_counts, stream=None) -> None:
     _check(load().dkv_get_counts(ctx, _ptr(host_counts), _stream(stream)), "dkv_get_counts")
 
@@ -266,7 +296,7 @@ def dkv_debug_withhold_tile(ctx: int, sweep: int, tile: int) -> None:
     _check(load().dkv_debug_withhold_tile(ctx, sweep, tile), "dkv_debug_withhold_tile")
 
 
-STEP_NAMES = ["score_stats", "score_emit", "select", "gather", "rebudget", "shrink", "other6", "other7"]
+STEP_NAMES = ["score_stats", "score_emit", "select", "gather", "rebudget", "shrink", "decode", "other7"]
 
 
 def dkv_profile(ctx: int, enable: bool) -> None:

@@ -9,11 +9,11 @@ namespace dkv {
 constexpr int kGatherRows = 4;      // rows per thread, all loads issued before the stores
 
 // Gather: dst[b,h,i] = src[b,h, i < n ? idx[i] : P + (i - n)], i < n + ws.  16 bytes per thread per row.
-// grid (row blocks, Bt*Hkv, 2 tensors).  n = kept positions per head (same for all heads); also records
-// held[b][layer] = n.
+// grid (row blocks, Bt*Hkv, 2 tensors).  n = kept positions per head (same for all heads), idx_stride = entries
+// per head in idx; also records held[b][layer] = n.
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v_src, uint4* __restrict__ kb,
-                   uint4* __restrict__ vb, const int* __restrict__ idx, int n, int S, int P, int ws,
+                   uint4* __restrict__ vb, const int* __restrict__ idx, int n, int idx_stride, int S, int P, int ws,
                    int row_stride /* rows per head in kb/vb */, int vec_per_row /* D*2/16 */,
                    int* __restrict__ held, int Hkv, int L, int layer) {
   const int bh = blockIdx.y;
@@ -28,7 +28,7 @@ gather_rows_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v_
   for (int j = 0; j < kGatherRows; ++j) {
     const int row = row0 + j * rows_per_pass;
     if (row < n + ws) {
-      const int from = row < n ? idx[(size_t)bh * n + row] : P + (row - n);
+      const int from = row < n ? idx[(size_t)bh * idx_stride + row] : P + (row - n);
       val[j] = src[(size_t)from * vec_per_row + c];
     }
   }

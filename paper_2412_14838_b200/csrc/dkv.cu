@@ -11,6 +11,7 @@
 #include "../../include/dkv.h"
 #include "common.cuh"
 #include "compact.cuh"
+#include "decode.cuh"
 #include "rebudget.cuh"
 #include "score_tc.cuh"
 #include "select.cuh"
@@ -59,7 +60,13 @@ struct dkv_ctx {
   int n_side;           // how many of them the pass uses
   cudaEvent_t ev_fork, ev_join[kSideStreams + 1], ev_update, ev_scored[DKV_MAX_LAYERS], ev_picked[DKV_MAX_LAYERS], ev_selected[DKV_MAX_LAYERS];
   // host state
-  uint8_t scored[DKV_MAX_LAYERS], selected[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
+  uint8_t scored[DKV_MAX_LAYERS], gathered[DKV_MAX_LAYERS], stale[DKV_MAX_LAYERS];
+  uint8_t selected[DKV_MAX_LAYERS];     // 1: by scores (dkv_select_topk), 2: by position (dkv_select_positions)
+  int sel_n[DKV_MAX_LAYERS];            // positions selected per head: Blc, or what dkv_select_positions kept
+  // decoding over the compressed cache (allocated on first use, grown on demand)
+  float* d_dec_scratch;
+  size_t dec_scratch_floats;
+  unsigned int* d_dec_tickets;          // [L][Bt*Hkv], zero between launches
   long long launches;
   // dkv_run_prefill_pass as a CUDA graph: captured on the first call with a set of pointers, replayed afterwards
   bool use_graph;
@@ -204,12 +211,13 @@ uint32_t make_idesc(int M, int N) {
 // key space from the end to the start: sweep 1 cut the same space into the same slices, so each CTA begins with
 // the keys that were streamed last and may still be in L2.
 bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, const void* const* k, float* scores_out,
-              int buf, tc::Maps* maps, tc::Params* p) {
+              int buf, tc::Maps* maps, tc::Params* p, const float* const* lse = nullptr) {
   const Shape& s = c->s;
   const int heads = s.Bt * s.Hkv;
   memset(maps, 0, sizeof *maps);                           // entries past nl are never read
   for (int i = 0; i < nl; ++i)
     if (!make_map(&maps->q[i], q[i], s.D, s.M, heads) || !make_map(&maps->k[i], k[i], s.D, s.S, heads)) return false;
+  if (lse) for (int i = 0; i < nl; ++i) maps->lse[i] = lse[i];
   p->S = s.S; p->P = s.P; p->ws = s.ws; p->M = s.M; p->D = s.D; p->heads = nl * heads; p->half = s.pool / 2;
   p->nl = nl; p->hpl = heads;
   p->back = (mode == tc::kEmit && c->emit_backward) ? 1 : 0;
@@ -228,7 +236,6 @@ bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, con
   p->mode = mode;
   p->out_scale = (c->cfg.flags & DKV_F_WINDOW_MEAN) ? 1.0f / (float)s.M : 1.0f;
   p->pool_avg = c->cfg.pool_kind == 1;
-  p->lse_in = nullptr;
   p->idesc = mode == tc::kStats ? make_idesc(128, 128) : make_idesc(128, p->nq16);
   return true;
 }
@@ -237,13 +244,13 @@ bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, con
 // `stats_layer` (if >= 0).  In the pass the emit layers are the ones the previous launch streamed.  `sbuf`, `ebuf`: statistics scratch of either job.
 int launch_score(dkv_ctx* c, int stats_layer, int sn, const void* const* sq, const void* const* sk, int sbuf,
                  int emit_layer, int en, const void* const* eq, const void* const* ek, int ebuf, float* scores_out,
-                 cudaStream_t st) {
+                 cudaStream_t st, const float* const* emit_lse = nullptr) {
   tc::Maps m0, m1;
   tc::Params j0, j1;
   memset(&j0, 0, sizeof j0); memset(&j1, 0, sizeof j1);
   memset(&m0, 0, sizeof m0); memset(&m1, 0, sizeof m1);
   j0.mode = j1.mode = tc::kNone;
-  if (emit_layer >= 0 && !make_job(c, tc::kEmit, emit_layer, en, eq, ek, scores_out, ebuf, &m0, &j0)) return DKV_ERR_CUDA;
+  if (emit_layer >= 0 && !make_job(c, tc::kEmit, emit_layer, en, eq, ek, scores_out, ebuf, &m0, &j0, emit_lse)) return DKV_ERR_CUDA;
   if (stats_layer >= 0 && !make_job(c, tc::kStats, stats_layer, sn, sq, sk, nullptr, sbuf, &m1, &j1)) return DKV_ERR_CUDA;
   ProfScope ps(c, stats_layer >= 0 ? DKV_STEP_SCORE_STATS : DKV_STEP_SCORE_EMIT, 1, st);
   tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(m0, m1, j0, j1);
@@ -258,8 +265,7 @@ int do_score_lse(dkv_ctx* c, int layer, const void* q, const void* k, const floa
   tc::Params job, none;
   memset(&job, 0, sizeof job); memset(&none, 0, sizeof none);
   none.mode = tc::kNone;
-  if (!make_job(c, tc::kEmit, layer, 1, &q, &k, scores_out, layer % 3, &maps, &job)) return DKV_ERR_CUDA;
-  job.lse_in = lse;
+  if (!make_job(c, tc::kEmit, layer, 1, &q, &k, scores_out, layer % 3, &maps, &job, &lse)) return DKV_ERR_CUDA;
   ProfScope ps(c, DKV_STEP_SCORE_EMIT, 1, st);
   tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(maps, maps, job, none);
   DKV_LAUNCHED(c);
@@ -302,6 +308,7 @@ int do_select(dkv_ctx* c, int layer, int* sorted_out, int* rank_out, cudaStream_
         sc, idx, sorted_out, rank_out, lh, s.P, s.Blc, c->sort_n, c->d_count, s.Hkv, s.L, layer);
   DKV_LAUNCHED(c);
   c->selected[layer] = 1;
+  c->sel_n[layer] = s.Blc;
   c->gathered[layer] = c->stale[layer] = 0;
   return DKV_OK;
 }
@@ -356,7 +363,7 @@ int do_gather(dkv_ctx* c, int layer, const void* k_src, const void* v_src, void*
   ProfScope ps(c, DKV_STEP_GATHER, 1, st);
   gather_rows_kernel<<<grid, 256, 0, st>>>(static_cast<const uint4*>(k_src), static_cast<const uint4*>(v_src),
                                            static_cast<uint4*>(kb), static_cast<uint4*>(vb),
-                                           c->d_idx + (size_t)layer * layer_idx(s), s.Blc, s.S, s.P, s.ws, s.rows, vec,
+                                           c->d_idx + (size_t)layer * layer_idx(s), c->sel_n[layer], s.Blc, s.S, s.P, s.ws, s.rows, vec,
                                            c->d_held, s.Hkv, s.L, layer);
   DKV_LAUNCHED(c);
   }
@@ -385,8 +392,9 @@ int do_reset(dkv_ctx* c, cudaStream_t st) {
 // fixed cost of a launch and of a job is paid once per group).  Everything that consumes a layer's scores (select,
 // gather, and every m layers rebudget + shrink) runs on side streams behind events, layers alternating between
 // two of them, so that it overlaps the scoring of the following groups.  `st` rejoins all of them at the end.
-int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* const* v, void* const* kb,
-            void* const* vb, cudaStream_t st) {
+// With `lse` (the window rows' log-denominators of every layer) sweep 1 is not needed: launch g runs sweep 2 of group g.
+int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* const* v, const float* const* lse,
+            void* const* kb, void* const* vb, cudaStream_t st) {
   const Shape& s = c->s;
   int rc = do_reset(c, st);
   if (rc) return rc;
@@ -408,11 +416,12 @@ int do_pass(dkv_ctx* c, const void* const* q, const void* const* k, const void* 
     done += n;
   }
   first[groups] = s.L;
-  for (int g = 0; g <= groups; ++g) {
-    const int sl = g < groups ? first[g] : -1, sn = g < groups ? first[g + 1] - first[g] : 0;
+  for (int g = lse ? 1 : 0; g <= groups; ++g) {
+    const int sl = g < groups && !lse ? first[g] : -1, sn = sl >= 0 ? first[g + 1] - first[g] : 0;
     const int e0 = g > 0 ? first[g - 1] : -1, en = g > 0 ? first[g] - first[g - 1] : 0;
     if ((rc = launch_score(c, sl, sn, sl >= 0 ? q + sl : nullptr, sl >= 0 ? k + sl : nullptr, g % 3, e0, en,
-                           e0 >= 0 ? q + e0 : nullptr, e0 >= 0 ? k + e0 : nullptr, (g + 2) % 3, nullptr, st)))
+                           e0 >= 0 ? q + e0 : nullptr, e0 >= 0 ? k + e0 : nullptr, (g + 2) % 3, nullptr, st,
+                           lse && e0 >= 0 ? lse + e0 : nullptr)))
       return rc;
     if (e0 < 0) continue;
     DKV_CUDA(c, cudaEventRecord(c->ev_scored[e0], st));
@@ -452,6 +461,7 @@ void free_all(dkv_ctx* c) {
   cudaFree(c->d_held); cudaFree(c->d_dbg); cudaFree(c->d_rb_state); cudaFree(c->d_rb_above); cudaFree(c->d_rb_hist1);
   cudaFree(c->d_rb_above2); cudaFree(c->d_rb_hist2); cudaFree(c->d_layer_hist);
   cudaFree(c->d_cand); cudaFree(c->d_cand_n); cudaFree(c->d_status); cudaFree(c->d_tc_stats);
+  cudaFree(c->d_dec_scratch); cudaFree(c->d_dec_tickets);
   for (int i = 0; i < kSideStreams; ++i) if (c->side[i]) cudaStreamDestroy(c->side[i]);
   if (c->hi) cudaStreamDestroy(c->hi);
   if (c->pass_exec) cudaGraphExecDestroy(c->pass_exec);
@@ -685,7 +695,7 @@ int dkv_select_topk(dkv_ctx* c, int32_t layer, int32_t* idx_out, int32_t* rank_o
 
 int dkv_rebudget(dkv_ctx* c, int32_t upto_layer, int32_t* counts_out, void* stream) {
   if (!c || upto_layer < 1 || upto_layer > c->s.L) return DKV_ERR_INVALID_ARG;
-  for (int i = 0; i < upto_layer; ++i) if (!c->scored[i] || !c->selected[i]) return DKV_ERR_STATE;
+  for (int i = 0; i < upto_layer; ++i) if (!c->scored[i] || c->selected[i] != 1) return DKV_ERR_STATE;
   return do_rebudget(c, upto_layer, counts_out, as_stream(stream));
 }
 
@@ -722,37 +732,41 @@ int dkv_compact_all(dkv_ctx* c, int32_t upto_layer, void* const* kb, void* const
   return do_shrink(c, 0, upto_layer, kb, vb, as_stream(stream));
 }
 
-int dkv_run_prefill_pass(dkv_ctx* c, const void* const* q_win, const void* const* k, const void* const* v,
-                         void* const* kb, void* const* vb, void* stream) {
+static int run_pass(dkv_ctx* c, const void* const* q_win, const void* const* k, const void* const* v,
+                    const float* const* lse, void* const* kb, void* const* vb, void* stream) {
   if (!c || !q_win || !k || !v || !kb || !vb) return DKV_ERR_INVALID_ARG;
   for (int l = 0; l < c->s.L; ++l) {
     if (!q_win[l] || !k[l] || !v[l] || !kb[l] || !vb[l]) return DKV_ERR_INVALID_ARG;
     if (!aligned16(q_win[l]) || !aligned16(k[l]) || !aligned16(v[l]) || !aligned16(kb[l]) || !aligned16(vb[l]))
       return DKV_ERR_INVALID_ARG;
+    if (lse && (!lse[l] || ((uintptr_t)lse[l] & 3))) return DKV_ERR_INVALID_ARG;
   }
   cudaStream_t st = as_stream(stream);
   cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
   if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
   // per-step profiling needs its events between the launches; a caller that is capturing gets the plain calls
-  if (!c->use_graph || c->prof_on || cap != cudaStreamCaptureStatusNone) return do_pass(c, q_win, k, v, kb, vb, st);
+  if (!c->use_graph || c->prof_on || cap != cudaStreamCaptureStatusNone) return do_pass(c, q_win, k, v, lse, kb, vb, st);
 
   std::vector<const void*> key;
-  key.reserve(5 * (size_t)c->s.L);
-  for (int l = 0; l < c->s.L; ++l) { key.push_back(q_win[l]); key.push_back(k[l]); key.push_back(v[l]); key.push_back(kb[l]); key.push_back(vb[l]); }
+  key.reserve(6 * (size_t)c->s.L);
+  for (int l = 0; l < c->s.L; ++l) {
+    key.push_back(q_win[l]); key.push_back(k[l]); key.push_back(v[l]); key.push_back(kb[l]); key.push_back(vb[l]);
+    key.push_back(lse ? lse[l] : nullptr);
+  }
   if (!c->pass_exec || *c->pass_key != key) {
     // first call with these buffers: record the whole pass (all streams of do_pass fork from and rejoin gstream)
     if (c->pass_exec) { cudaGraphExecDestroy(c->pass_exec); c->pass_exec = nullptr; }
     const long long before = c->launches;
     cudaGraph_t graph = nullptr;
     DKV_CUDA(c, cudaStreamBeginCapture(c->gstream, cudaStreamCaptureModeThreadLocal));
-    const int rc = do_pass(c, q_win, k, v, kb, vb, c->gstream);
+    const int rc = do_pass(c, q_win, k, v, lse, kb, vb, c->gstream);
     const cudaError_t e = cudaStreamEndCapture(c->gstream, &graph);
     if (rc != DKV_OK || e != cudaSuccess || !graph) {
       if (graph) cudaGraphDestroy(graph);
       cudaGetLastError();
       c->launches = before;
       c->use_graph = false;                         // not capturable here: run the plain calls from now on
-      return do_pass(c, q_win, k, v, kb, vb, st);
+      return do_pass(c, q_win, k, v, lse, kb, vb, st);
     }
     c->pass_launches = c->launches - before;
     c->launches = before;
@@ -761,7 +775,7 @@ int dkv_run_prefill_pass(dkv_ctx* c, const void* const* q_win, const void* const
     if (ei != cudaSuccess) {
       cudaGetLastError();
       c->pass_exec = nullptr; c->use_graph = false;
-      return do_pass(c, q_win, k, v, kb, vb, st);
+      return do_pass(c, q_win, k, v, lse, kb, vb, st);
     }
     *c->pass_key = key;
   }
@@ -771,8 +785,19 @@ int dkv_run_prefill_pass(dkv_ctx* c, const void* const* q_win, const void* const
   DKV_CUDA(c, cudaEventRecord(c->ev_gjoin, c->gstream));
   DKV_CUDA(c, cudaStreamWaitEvent(st, c->ev_gjoin, 0));
   c->launches += c->pass_launches;
-  for (int l = 0; l < c->s.L; ++l) { c->scored[l] = c->selected[l] = c->gathered[l] = 1; c->stale[l] = 0; }
+  for (int l = 0; l < c->s.L; ++l) { c->scored[l] = c->selected[l] = c->gathered[l] = 1; c->stale[l] = 0; c->sel_n[l] = c->s.Blc; }
   return DKV_OK;
+}
+
+int dkv_run_prefill_pass(dkv_ctx* c, const void* const* q_win, const void* const* k, const void* const* v,
+                         void* const* kb, void* const* vb, void* stream) {
+  return run_pass(c, q_win, k, v, nullptr, kb, vb, stream);
+}
+
+int dkv_run_prefill_pass_lse(dkv_ctx* c, const void* const* q_win, const void* const* k, const void* const* v,
+                             const float* const* lse, void* const* kb, void* const* vb, void* stream) {
+  if (!lse) return DKV_ERR_INVALID_ARG;
+  return run_pass(c, q_win, k, v, lse, kb, vb, stream);
 }
 
 int dkv_run_prefill_pass_host(dkv_ctx* c, const void* const* q_win, const void* const* k, const void* const* v,
@@ -811,6 +836,85 @@ int dkv_run_prefill_pass_host(dkv_ctx* c, const void* const* q_win, const void* 
     DKV_CUDA(c, cudaMemcpyAsync(counts_out, c->d_count, sizeof(int) * s.Bt * s.L, cudaMemcpyDeviceToHost, st));
   DKV_CUDA(c, cudaStreamSynchronize(cp));
   DKV_CUDA(c, cudaStreamSynchronize(st));
+  return DKV_OK;
+}
+
+int dkv_apply_policy(dkv_ctx* c, int32_t policy, int32_t* counts_out, void* stream) {
+  if (!c || (policy != DKV_POLICY_UNIFORM && policy != DKV_POLICY_PYRAMID)) return DKV_ERR_INVALID_ARG;
+  const Shape& s = c->s;
+  for (int i = 0; i < s.L; ++i) if (!c->selected[i]) return DKV_ERR_STATE;
+  policy_counts_kernel<<<(s.Bt * s.L + 127) / 128, 128, 0, as_stream(stream)>>>(c->d_count, counts_out, s.Bt, s.L, s.N, policy);
+  DKV_LAUNCHED(c);
+  for (int i = 0; i < s.L; ++i) if (!c->gathered[i]) c->stale[i] = 1;
+  return DKV_OK;
+}
+
+int dkv_select_positions(dkv_ctx* c, int32_t layer, int32_t n_sink, int32_t n_recent, void* stream) {
+  int rc = check_layer(c, layer);
+  if (rc) return rc;
+  const Shape& s = c->s;
+  if (n_sink < 0 || n_recent < 0) return DKV_ERR_INVALID_ARG;
+  if (n_sink > s.P) n_sink = s.P;
+  if (n_recent > s.P) n_recent = s.P;
+  const int first_recent = s.P - n_recent > n_sink ? s.P - n_recent : n_sink;
+  const int n = n_sink + (s.P - first_recent);
+  if (n > s.Blc) return DKV_ERR_INVALID_ARG;
+  {
+    const dim3 grid((n + 255) / 256 > 0 ? (n + 255) / 256 : 1, s.Bt * s.Hkv);
+    positions_kernel<<<grid, 256, 0, as_stream(stream)>>>(c->d_idx + (size_t)layer * layer_idx(s), c->d_count, s.P, s.Blc, n_sink,
+                                                         first_recent, n, s.Hkv, s.L, layer);
+    DKV_LAUNCHED(c);
+  }
+  c->selected[layer] = 2;
+  c->sel_n[layer] = n;
+  c->gathered[layer] = c->stale[layer] = 0;
+  return DKV_OK;
+}
+
+int dkv_decode_attend(dkv_ctx* c, int32_t layer0, int32_t n_layers, int32_t nq, const void* const* q_dec,
+                      const void* const* kb, const void* const* vb, float* const* out, void* stream) {
+  if (!c || !q_dec || !kb || !vb || !out) return DKV_ERR_INVALID_ARG;
+  const Shape& s = c->s;
+  if (layer0 < 0 || n_layers < 1 || layer0 + n_layers > s.L || nq < 1 || (long long)nq * s.G > 64) return DKV_ERR_INVALID_ARG;
+  for (int i = 0; i < n_layers; ++i) {
+    if (!q_dec[i] || !kb[i] || !vb[i] || !out[i]) return DKV_ERR_INVALID_ARG;
+    if (!aligned16(q_dec[i]) || !aligned16(kb[i]) || !aligned16(vb[i]) || !aligned16(out[i])) return DKV_ERR_INVALID_ARG;
+    if (!c->gathered[layer0 + i]) return DKV_ERR_STATE;
+  }
+  cudaStream_t st = as_stream(stream);
+  const int BH = s.Bt * s.Hkv, GQ = s.G * nq;
+  if (!c->d_dec_tickets) {
+    DKV_CUDA(c, cudaMalloc(&c->d_dec_tickets, sizeof(unsigned int) * s.L * BH));
+    DKV_CUDA(c, cudaMemset(c->d_dec_tickets, 0, sizeof(unsigned int) * s.L * BH));
+  }
+  for (int l0 = 0; l0 < n_layers; l0 += kDecMaxLayers) {
+    const int nl = n_layers - l0 < kDecMaxLayers ? n_layers - l0 : kDecMaxLayers;
+    // enough thread blocks to fill the GPU a few times over, each with at least a few dozen rows
+    int splits = (4 * c->n_sms + BH * nl - 1) / (BH * nl);
+    const int most = (s.rows + 31) / 32;
+    if (splits > most) splits = most;
+    if (splits > 64) splits = 64;
+    if (splits < 1) splits = 1;
+    const size_t need = (size_t)nl * BH * splits * GQ * (s.D + 2);
+    if (need > c->dec_scratch_floats) {
+      if (c->d_dec_scratch) { DKV_CUDA(c, cudaDeviceSynchronize()); cudaFree(c->d_dec_scratch); c->d_dec_scratch = nullptr; c->dec_scratch_floats = 0; }
+      DKV_CUDA(c, cudaMalloc(&c->d_dec_scratch, need * sizeof(float)));
+      c->dec_scratch_floats = need;
+    }
+    DecodePtrs ptrs;
+    memset(&ptrs, 0, sizeof ptrs);
+    for (int i = 0; i < nl; ++i) { ptrs.q[i] = q_dec[l0 + i]; ptrs.kb[i] = kb[l0 + i]; ptrs.vb[i] = vb[l0 + i]; ptrs.out[i] = out[l0 + i]; }
+    const dim3 grid(splits, BH, nl);
+    const float scale2 = kLog2e / sqrtf((float)s.D);
+    ProfScope ps(c, DKV_STEP_DECODE, 1, st);
+    if (s.D == 128)
+      decode_attend_kernel<128><<<grid, kDecThreads, 0, st>>>(ptrs, layer0 + l0, c->d_held, s.Hkv, s.G, nq, s.L, s.ws, s.rows, scale2,
+                                                             c->d_dec_scratch, c->d_dec_tickets + (size_t)(layer0 + l0) * BH);
+    else
+      decode_attend_kernel<64><<<grid, kDecThreads, 0, st>>>(ptrs, layer0 + l0, c->d_held, s.Hkv, s.G, nq, s.L, s.ws, s.rows, scale2,
+                                                            c->d_dec_scratch, c->d_dec_tickets + (size_t)(layer0 + l0) * BH);
+    DKV_LAUNCHED(c);
+  }
   return DKV_OK;
 }
 

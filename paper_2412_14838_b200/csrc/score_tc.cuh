@@ -59,7 +59,6 @@ struct Params {
   int mode;                // kNone: nothing to do
   float out_scale;         // sweep 2: factor on the raw scores before pooling (1, or 1/(ws*G) for the window mean)
   int pool_avg;            // sweep 2: 0 = max-pool, 1 = average over the neighbours that exist
-  const float* lse_in;     // sweep 2: caller's natural-log normalisers [heads][M] (then sweep 1 never ran), or null
   int nl;                  // layers this job covers (1..kMaxGroup); `heads` counts the heads of all of them
   int hpl;                 // heads per layer
   int back;                // sweep 2: 1 = every CTA walks its slice from the end to the start, so that it begins
@@ -72,6 +71,8 @@ struct Params {
 constexpr int kMaxGroup = 8;               // layers one job may cover
 struct Maps {                              // tensor maps of a job's layers, in storage order
   CUtensorMap q[kMaxGroup], k[kMaxGroup];
+  const float* lse[kMaxGroup];             // sweep 2: the caller's natural-log normalisers [heads per layer][M] of each
+                                           // layer (then sweep 1 never ran for the job), or null
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -497,8 +498,9 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
             const int c_lo = tile_owner((long long)nb * p.tph, total, p.stats_grid);
             const int c_hi = tile_owner((long long)(nb + 1) * p.tph - 1, total, p.stats_grid);
             float lse = INFINITY;
-            if (p.lse_in) {
-              if (sid < p.M) lse = p.lse_in[(size_t)nb * p.M + sid] * kLog2e;
+            const float* lse_in = (jb ? maps1 : maps0).lse[nb / p.hpl];
+            if (lse_in) {
+              if (sid < p.M) lse = lse_in[(size_t)(nb % p.hpl) * p.M + sid] * kLog2e;
             } else if (sid < p.M) {
               float m = -INFINITY;
               for (int c = 0; c <= c_hi - c_lo; ++c) m = fmaxf(m, p.stats[((size_t)nb * p.slots + c) * p.m_stride + sid].x);

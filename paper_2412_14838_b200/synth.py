@@ -24,7 +24,7 @@ import numpy as np
 
 BASE_SEED = 20241214
 
-_T_Q, _T_K, _T_V, _T_MU, _T_AUX, _T_SCORES = 1, 2, 3, 4, 5, 6
+_T_Q, _T_K, _T_V, _T_MU, _T_AUX, _T_SCORES, _T_QDEC = 1, 2, 3, 4, 5, 6, 7
 
 
 @dataclass(frozen=True)
@@ -192,6 +192,18 @@ def layer_inputs(w: Workload, layer: int, seed: int = BASE_SEED, want_v: bool = 
     if want_v:
         out["v"] = f32_to_bf16_bits(_normal(gv, (Bt, Hkv, S, D)))
     return out
+
+
+def decode_queries(w: Workload, layer: int, nq: int = 1, seed: int = BASE_SEED) -> np.ndarray:
+    """Queries of ``nq`` newly generated tokens per sample for one layer, bf16 bit patterns [Bt, Hq, nq, D]:
+    N(0,1) plus, for the recipes that have one, the layer's mean query direction of the head group (so that the
+    decode step attends to the same sinks and planted keys as the window queries did)."""
+    g = _rng(seed, w.cid, _T_QDEC, layer)
+    q = _normal(g, (w.Bt, w.Hq, nq, w.D))
+    if w.recipe != "iid":
+        mu = _normal(_rng(seed, w.cid, _T_MU, layer), (w.Bt, w.Hkv, w.D))
+        q = q + np.repeat(mu, w.G, axis=1)[:, :, None, :]
+    return f32_to_bf16_bits(q)
 
 
 def pooled_like_scores(shape, pool: int, seed: int, tie_fraction: float = 0.0) -> np.ndarray:

@@ -1,0 +1,159 @@
+"""GPU parity of the steps around Algorithm 1's loop: decoding over the compressed, ragged cache (Section 4.3),
+the fixed-pattern budget policies of the methods the paper compares with (Section 5.1), and the pass scored in
+one sweep from the window rows' log-denominators.  Everything goes through the C ABI; expected values come
+from the oracle run on the same seeded inputs (never from the GPU)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dynamickv as O
+from paper_2412_14838_b200 import binding as B
+from paper_2412_14838_b200 import build, synth
+from tests import _util as U
+from tests.test_gpu_pass import GpuPass, check_decode, check_properties, compare_full, dev
+
+pytestmark = pytest.mark.gpu
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    B.load()
+
+
+def oracle_pass(w, host, **kw):
+    fn = lambda l: {"q": synth.bf16_bits_to_f64(host[l]["q"]), "k": synth.bf16_bits_to_f64(host[l]["k"]),
+                    "k_rows": host[l]["k"], "v_rows": host[l]["v"]}
+    return O.run_prefill_pass(fn, w.L, ws=w.ws, pool=w.pool, N=w.N, Bl=w.Bl, m=w.m, **kw)
+
+
+@pytest.mark.parametrize("name,nq,per_call", [("tiny", 1, 4), ("tiny", 3, 1), ("ragdec", 2, 5), ("ragdec", 5, 2)])
+def test_decode_attention_matches_oracle(name, nq, per_call):
+    w = synth.WORKLOADS.get(name) or synth.Workload("ragdec", 91, L=5, Hq=6, Hkv=2, D=128, Bt=2, S=1700, ws=8, pool=3,
+                                                    N=40, Bl=100, m=2, recipe="sink")
+    g = GpuPass(w).run()
+    try:
+        ref = oracle_pass(w, g.host)
+        assert (g.counts == ref["counts"]).all()
+        worst = check_decode(g, ref, nq, per_call)
+        print(f"[{w.name}] decode nq={nq}, {per_call} layers per call: worst error {worst:.2e}")
+    finally:
+        g.close()
+
+
+def test_decode_arguments_are_checked():
+    w = synth.WORKLOADS["tiny"]
+    g = GpuPass(w)
+    try:
+        q = [dev(synth.decode_queries(w, l)) for l in range(w.L)]
+        out = [torch.zeros((w.Bt, w.Hq, 1, w.D), dtype=torch.float32, device="cuda") for _ in range(w.L)]
+        with pytest.raises(B.DkvError) as e:                     # nothing gathered yet
+            B.dkv_decode_attend(g.h, 0, 1, 1, q[:1], g.kb[:1], g.vb[:1], out[:1])
+        assert e.value.code == B.DKV_ERR_STATE
+        g.run()
+        with pytest.raises(B.DkvError) as e:
+            B.dkv_decode_attend(g.h, 2, 3, 1, q[:3], g.kb[:3], g.vb[:3], out[:3])     # past the last layer
+        assert e.value.code == B.DKV_ERR_INVALID_ARG
+        with pytest.raises(B.DkvError) as e:
+            B.dkv_decode_attend(g.h, 0, 1, 100, q[:1], g.kb[:1], g.vb[:1], out[:1])    # too many queries
+        assert e.value.code == B.DKV_ERR_INVALID_ARG
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("policy,name", [(B.DKV_POLICY_UNIFORM, "uniform"), (B.DKV_POLICY_PYRAMID, "pyramid")])
+def test_budget_policies_bit_exact(policy, name):
+    # injected scores with ties; L odd so that the pyramid's floors towards minus infinity are exercised
+    w = synth.Workload("pol", 92, L=7, Hq=4, Hkv=2, D=64, Bt=2, S=900, ws=8, pool=5, N=21, Bl=48, m=100, recipe="iid")
+    sc = [synth.pooled_like_scores((w.Bt, w.Hkv, w.P), w.pool, seed=100 + l, tie_fraction=0.2) for l in range(w.L)]
+    host = [synth.layer_inputs(w, l) for l in range(w.L)]
+    k, v = [dev(t["k"]) for t in host], [dev(t["v"]) for t in host]
+    shape = (w.Bt, w.Hkv, w.Blc + w.ws, w.D)
+    kb = [torch.zeros(shape, dtype=torch.int16, device="cuda") for _ in range(w.L)]
+    vb = [torch.zeros(shape, dtype=torch.int16, device="cuda") for _ in range(w.L)]
+    h = B.dkv_create(B.config_of(w))
+    try:
+        with pytest.raises(B.DkvError) as e:
+            B.dkv_apply_policy(h, policy)                         # nothing selected yet
+        assert e.value.code == B.DKV_ERR_STATE
+        for l in range(w.L):
+            B.dkv_set_scores(h, l, torch.from_numpy(sc[l]).cuda())
+            B.dkv_select_topk(h, l)
+            if l < w.L - 2:
+                B.dkv_compact(h, l, k[l], v[l], kb[l], vb[l])
+        counts_dev = torch.zeros((w.Bt, w.L), dtype=torch.int32, device="cuda")
+        B.dkv_apply_policy(h, policy, counts_dev)
+        B.dkv_compact_all(h, w.L - 2, kb[:w.L - 2], vb[:w.L - 2])
+        for l in range(w.L - 2, w.L):                             # gathered after the policy: picks the count up
+            B.dkv_compact(h, l, k[l], v[l], kb[l], vb[l])
+        torch.cuda.synchronize()
+        want = np.minimum(O.policy_counts(name, w.L, w.N), w.Blc)
+        assert (counts_dev.cpu().numpy() == want[None, :]).all()
+        for l in range(w.L):
+            n = int(want[l])
+            got_k, got_v = kb[l].cpu().numpy().view(np.uint16), vb[l].cpu().numpy().view(np.uint16)
+            for b in range(w.Bt):
+                for hh in range(w.Hkv):
+                    sel = O.select_topk(sc[l][b, hh].astype(np.float64), n)
+                    order = sel["idx"][np.argsort(sel["rank"], kind="stable")]          # buffer order: by rank
+                    for got, rows in ((got_k, host[l]["k"]), (got_v, host[l]["v"])):
+                        assert (got[b, hh, :n] == rows[b, hh][order]).all(), f"kept rows differ l={l}"
+                        assert (got[b, hh, n:n + w.ws] == rows[b, hh][w.P:]).all(), f"window rows differ l={l}"
+    finally:
+        B.dkv_destroy(h)
+
+
+def test_sinks_plus_recent_selection():
+    w = synth.Workload("sinks", 93, L=2, Hq=4, Hkv=2, D=128, Bt=2, S=700, ws=8, pool=3, N=20, Bl=40, m=1, recipe="sink")
+    host = [synth.layer_inputs(w, l) for l in range(w.L)]
+    h = B.dkv_create(B.config_of(w))
+    try:
+        for l, (a, r) in enumerate([(4, 16), (0, 40)]):
+            B.dkv_select_positions(h, l, a, r)
+            kb = torch.zeros((w.Bt, w.Hkv, w.Blc + w.ws, w.D), dtype=torch.int16, device="cuda")
+            vb = torch.zeros_like(kb)
+            ln = torch.zeros((w.Bt, w.Hkv), dtype=torch.int32, device="cuda")
+            B.dkv_compact(h, l, dev(host[l]["k"]), dev(host[l]["v"]), kb, vb, ln)
+            srt = torch.zeros((w.Bt, w.Hkv, w.Blc), dtype=torch.int32, device="cuda")
+            B.dkv_kept_sorted(h, l, srt)
+            torch.cuda.synchronize()
+            pos = O.positions_sinks_recent(w.P, a, r)
+            assert (ln.cpu().numpy() == len(pos) + w.ws).all()
+            assert (srt.cpu().numpy()[:, :, :len(pos)] == pos[None, None, :]).all()
+            got = kb.cpu().numpy().view(np.uint16)
+            for b in range(w.Bt):
+                for hh in range(w.Hkv):
+                    assert (got[b, hh, :len(pos) + w.ws] == O.gather_rows(host[l]["k"][b, hh], pos, w.ws)).all()
+        with pytest.raises(B.DkvError) as e:
+            B.dkv_select_positions(h, 0, 30, 30)                   # 60 positions do not fit Bl = 40
+        assert e.value.code == B.DKV_ERR_INVALID_ARG
+        with pytest.raises(B.DkvError) as e:
+            B.dkv_rebudget(h, 1)                                   # a layer selected by position has no scores to rank
+        assert e.value.code == B.DKV_ERR_STATE
+    finally:
+        B.dkv_destroy(h)
+
+
+def window_lse_dev(w, host):
+    lse = []
+    for l in range(w.L):
+        q, k = synth.bf16_bits_to_f64(host[l]["q"]), synth.bf16_bits_to_f64(host[l]["k"])
+        lse.append(torch.from_numpy(O.window_lse(q, k, w.ws).astype(np.float32)).cuda())
+    return lse
+
+
+@pytest.mark.parametrize("name", ["tiny", "mistral8k", "raglse"])
+def test_pass_scored_from_log_denominators_matches_oracle(name):
+    w = synth.WORKLOADS.get(name) or synth.Workload("raglse", 94, L=5, Hq=6, Hkv=2, D=128, Bt=2, S=1500, ws=8, pool=3,
+                                                    N=24, Bl=60, m=2, recipe="sink")
+    g = GpuPass(w)
+    try:
+        lse = window_lse_dev(w, g.host)                            # fp32 values, as an attention kernel would return
+        g.run_with = lambda: B.dkv_run_prefill_pass_lse(g.h, g.q, g.k, g.v, lse, g.kb, g.vb)
+        g.run()
+        check_properties(g)
+        near = compare_full(g)          # the oracle's two-sweep pass: the same quantity up to the rounding of lse
+        assert near <= 8
+        g.run()                          # replayed graph
+        check_properties(g)
+    finally:
+        g.close()

@@ -44,9 +44,13 @@ class GpuPass:
         self.kb = [torch.zeros(shape, dtype=torch.int16, device="cuda") for _ in range(w.L)]
         self.vb = [torch.zeros(shape, dtype=torch.int16, device="cuda") for _ in range(w.L)]
         self.h = B.dkv_create(B.config_of(w, pool_kind, flags))
+        self.run_with = None               # another way to run the pass (same results expected), or None
 
     def run(self):
-        B.dkv_run_prefill_pass(self.h, self.q, self.k, self.v, self.kb, self.vb)
+        if self.run_with is not None:
+            self.run_with()
+        else:
+            B.dkv_run_prefill_pass(self.h, self.q, self.k, self.v, self.kb, self.vb)
         torch.cuda.synchronize()
         w = self.w
         self.counts = np.zeros((w.Bt, w.L), dtype=np.int32)
@@ -145,6 +149,33 @@ def compare_full(g: GpuPass, verbose_name=""):
     return near
 
 
+DECODE_TOL = 1e-3        # max |gpu - oracle| over a head's output vector, relative to that vector's largest entry
+
+
+def check_decode(g, ref, nq, layers_per_call):
+    """dkv_decode_attend against the oracle's attention over the ORACLE's final buffers (row order differs between
+    the two sides, which attention does not see)."""
+    w = g.w
+    qd = [synth.decode_queries(w, l, nq) for l in range(w.L)]
+    dq = [dev(x) for x in qd]
+    out = [torch.full((w.Bt, w.Hq, nq, w.D), float("nan"), dtype=torch.float32, device="cuda") for _ in range(w.L)]
+    for l0 in range(0, w.L, layers_per_call):
+        n = min(layers_per_call, w.L - l0)
+        B.dkv_decode_attend(g.h, l0, n, nq, dq[l0:l0 + n], g.kb[l0:l0 + n], g.vb[l0:l0 + n], out[l0:l0 + n])
+    torch.cuda.synchronize()
+    worst = 0.0
+    for l in range(w.L):
+        kb = [[synth.bf16_bits_to_f64(ref["kb"][l][b][h]) for h in range(w.Hkv)] for b in range(w.Bt)]
+        vb = [[synth.bf16_bits_to_f64(ref["vb"][l][b][h]) for h in range(w.Hkv)] for b in range(w.Bt)]
+        want = O.decode_attention(synth.bf16_bits_to_f64(qd[l]), kb, vb, ref["counts"][:, l] + w.ws)
+        got = out[l].cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all(), f"layer {l}: outputs never written"
+        err = np.abs(got - want).max(axis=-1) / np.abs(want).max(axis=-1)
+        worst = max(worst, float(err.max()))
+    assert worst <= DECODE_TOL, f"decode attention off by {worst:.2e}"
+    return worst
+
+
 def replay_counts(g: GpuPass):
     """Algorithm 1's budget updates replayed by the oracle on the scores the pass itself stored (fp32, widened
     exactly): the per-layer counts must then agree bit for bit, whatever the rounding of the scores was."""
@@ -222,6 +253,54 @@ def test_pass_is_the_same_however_the_layers_are_grouped(group, taper, streams, 
         g.close()
 
 
+def policy_retention(g: GpuPass):
+    """Needle retention of the fixed-pattern budgets beside DynamicKV's, GPU against oracle: the policies run through
+    the library's select / policy kernels on the pass's own scores in a second context; the oracle takes its own
+    scores and schedules."""
+    w = g.w
+    mask = synth.needle_token_mask(w)
+    total = float(mask.sum())
+    h = B.dkv_create(B.config_of(w))
+    try:
+        for l in range(w.L):
+            B.dkv_set_scores(h, l, B.dkv_layer_views(g.h, l)[0])
+            B.dkv_select_topk(h, l)
+        torch.cuda.synchronize()
+        first = [B.read_device_i32(h, B.dkv_layer_views(h, l)[1], (w.Bt, w.Hkv, w.Blc)) for l in range(w.L)]
+        rows = {"dynamickv": (needle_retention(w, lambda l, hh: np.sort(g.kept(l)[1][0, hh, :int(g.counts[0, l])]), g.counts),
+                              needle_retention(w, lambda l, hh: g.ref["idx"][l][0][hh], g.ref["counts"]))}
+        for pol, pname in ((B.DKV_POLICY_UNIFORM, "uniform"), (B.DKV_POLICY_PYRAMID, "pyramid")):
+            cd = torch.zeros((w.Bt, w.L), dtype=torch.int32, device="cuda")
+            hp = B.dkv_create(B.config_of(w))
+            try:
+                for l in range(w.L):
+                    B.dkv_set_scores(hp, l, B.dkv_layer_views(g.h, l)[0])
+                    B.dkv_select_topk(hp, l)
+                B.dkv_apply_policy(hp, pol, cd)
+                torch.cuda.synchronize()
+            finally:
+                B.dkv_destroy(hp)
+            c_gpu = cd.cpu().numpy()
+            c_ora = np.minimum(np.array(O.policy_counts(pname, w.L, w.N)), w.Blc)[None, :]
+            assert (c_gpu == c_ora).all()
+            gpu = needle_retention(w, lambda l, hh: first[l][0, hh], c_gpu)             # buffer order: a prefix is the top-c
+            ora = needle_retention(w, lambda l, hh: O.select_topk(g.ref["score"][l][0, hh], int(c_ora[0, l]))["idx"], c_ora)
+            rows[pname] = (gpu, ora)
+        n_sink, n_recent = 4, w.N - 4
+        B.dkv_select_positions(h, 0, n_sink, n_recent)
+        pos_gpu = B.read_device_i32(h, B.dkv_layer_views(h, 0)[1], (w.Bt, w.Hkv, w.Blc))[0, 0, :w.N]
+        pos_ora = O.positions_sinks_recent(w.P, n_sink, n_recent)
+        assert (pos_gpu == pos_ora).all()
+        rows["sinks+recent"] = ([float(mask[pos_gpu].sum() / total)] * w.L, [float(mask[pos_ora].sum() / total)] * w.L)
+        for pname, (gpu, ora) in rows.items():
+            lay = slice(7, 24)                                       # the layers that carry the needles
+            print(f"[needle32k] policy {pname:13s}: needle tokens retained in layers 8-24, mean over layers: "
+                  f"GPU {np.mean(gpu[lay]):.3f}  oracle {np.mean(ora[lay]):.3f}; budget {w.N} tokens/head/layer on average")
+            assert np.allclose(gpu, ora, atol=2.0 / total), f"{pname}: retention differs from the oracle's"
+    finally:
+        B.dkv_destroy(h)
+
+
 FULL = ["mistral32k", "llama16k_b4", "needle32k", "qwen16k"]
 
 
@@ -262,6 +341,12 @@ def test_full_size_pass_whole_oracle(name):
     try:
         near = compare_full(g)
         assert near <= 8, "implausibly many near-ties"
+        if (g.counts == g.ref["counts"]).all():
+            # the decode step over the final ragged buffers, all layers in one launch and layer by layer
+            worst = max(check_decode(g, g.ref, 1, w.L), check_decode(g, g.ref, 2, 1))
+            print(f"[{name}] decode attention over the compressed cache: worst error {worst:.2e}")
+        if name == "needle32k":
+            policy_retention(g)
         if name == "needle32k":
             kept = {l: g.kept(l)[0] for l in range(w.L)}
             gpu = needle_retention(w, lambda l, h: kept[l][0, h], g.counts)
