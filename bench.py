@@ -124,13 +124,14 @@ def run_reference(args, w):
     for _ in range(args.steps):
         dt, cores = oracle_sample(w, layers, inputs)
         times.append(dt)
-    per_step = float(np.mean(times)) * w.L / layers
-    value = w.Bt * w.S / per_step
+    measured = float(np.mean(times))                 # seconds one step really took
+    per_pass = measured * w.L / layers               # the same rate over all L layers
+    value = w.Bt * w.S / per_pass
     base = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"each step = layers 0..{layers - 1} of {w.L} of workload {w.name} "
-                      f"({float(np.mean(times)):.2f} s), scaled by {w.L}/{layers} to a whole pass"}
+            "sample": f"each step = layers 0..{layers - 1} of {w.L} of workload {w.name} ({measured:.2f} s measured, "
+                      f"ms_per_step is that time); value = tokens of a whole pass / (step time x {w.L}/{layers})"}
     return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": measured * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": workload_config(w), "cpu_baseline": base,
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -264,8 +265,16 @@ def run_gpu(args, w):
     for _ in range(args.warmup):
         one_pass()
     barrier()
-    launches0 = B.dkv_launch_count(ctx)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # a short burst first (the clocks have not yet met the power cap), reported beside the sustained figure
+    burst_steps = min(20, args.steps)
+    ev0.record(stream)
+    for _ in range(burst_steps):
+        one_pass()
+    ev1.record(stream)
+    barrier()
+    burst_ms = max_over_ranks(ev0.elapsed_time(ev1)) / burst_steps
+    launches0 = B.dkv_launch_count(ctx)
     with ClockSampler(local) as clocks:
         ev0.record(stream)
         for _ in range(args.steps):
@@ -337,7 +346,55 @@ def run_gpu(args, w):
         one_sweep = {"api": "dkv_score_lse", "avg_launch_ms": one_ms, "algorithmic_bytes_per_launch": k_bytes,
                      "achieved": k_bytes / (one_ms * 1e-3) / 1e9, "unit": "GB/s",
                      "frac": k_bytes / (one_ms * 1e-3) / 1e9 / peak}
+
+    # the pass scored in one sweep (dkv_run_prefill_pass_lse), normalisers prepared outside the timed region;
+    # reported beside the headline, never part of it
+    one_sweep_pass = None
+    if one_sweep is not None:
+        def lse_pass():
+            B.dkv_run_prefill_pass_lse(ctx, q, k, v, lse, kb, vb, stream)
+        for _ in range(3):
+            lse_pass()
+        barrier()
+        ev0.record(stream)
+        for _ in range(prof_steps):
+            lse_pass()
+        ev1.record(stream)
+        barrier()
+        lp_ms = max_over_ranks(ev0.elapsed_time(ev1)) / prof_steps
+        one_sweep_pass = {"api": "dkv_run_prefill_pass_lse", "ms_per_step": lp_ms, "steps": prof_steps,
+                          "value": whole_job_value(tokens, world, lp_ms * 1e-3), "unit": UNIT,
+                          "whole_pass_frac_of_measured_peak": w.algorithmic_bytes() / (lp_ms * 1e-3) / 1e9 / peak}
         del lse
+
+    # decoding over the compressed cache the pass leaves behind: one new query per sample, all layers in one
+    # launch, then layer by layer; algorithmic bytes = the valid K and V rows, once
+    one_pass()
+    barrier()
+    counts_now = np.zeros((w.Bt, w.L), dtype=np.int32)
+    B.dkv_get_counts(ctx, counts_now)
+    dq = [to_dev(synth.decode_queries(w, l)) for l in range(w.L)]
+    dout = [torch.zeros((w.Bt, w.Hq, 1, w.D), dtype=torch.float32, device="cuda") for _ in range(w.L)]
+    dec_bytes = int((counts_now.astype(np.int64) + w.ws).sum()) * w.Hkv * w.D * 2 * 2
+    dec = {}
+    for label, per_call in (("all_layers_one_launch", w.L), ("layer_by_layer", 1)):
+        def dec_step():
+            for l0 in range(0, w.L, per_call):
+                B.dkv_decode_attend(ctx, l0, per_call, 1, dq[l0:l0 + per_call], kb[l0:l0 + per_call], vb[l0:l0 + per_call],
+                                    dout[l0:l0 + per_call], stream)
+        for _ in range(3):
+            dec_step()
+        barrier()
+        ev0.record(stream)
+        for _ in range(prof_steps):
+            dec_step()
+        ev1.record(stream)
+        barrier()
+        d_ms = max_over_ranks(ev0.elapsed_time(ev1)) / prof_steps
+        dec[label] = {"ms": d_ms, "achieved": dec_bytes / (d_ms * 1e-3) / 1e9, "frac": dec_bytes / (d_ms * 1e-3) / 1e9 / peak}
+    decode = {"api": "dkv_decode_attend", "queries_per_sample": 1, "algorithmic_bytes": dec_bytes, "unit": "GB/s",
+              "bound": "hbm", "peak": peak, "note": "the buffers of a pass fit L2, so repeated calls are served from it",
+              **dec}
 
     # end to end: host buffers in, compacted buffers + counts out, copies inside the timed region
     e2e = None
@@ -368,9 +425,14 @@ def run_gpu(args, w):
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
-               "config": dict(workload_config(w), parallelism=f"{world} independent replica(s)"),
+               "config": workload_config(w), "parallelism": f"{world} independent replica(s)",
                "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-               "one_sweep_scoring": one_sweep, "cpu_baseline": base}
+               "burst": {"steps": burst_steps, "ms_per_step": burst_ms,
+                         "value": whole_job_value(tokens, world, burst_ms * 1e-3),
+                         "note": "the first timed steps, before the clocks meet the power cap; `value` is the "
+                                 "sustained figure over all `steps`"},
+               "one_sweep_scoring": one_sweep, "one_sweep_pass": one_sweep_pass, "decode_attention": decode,
+               "cpu_baseline": base}
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
