@@ -21,6 +21,7 @@ constexpr int kDecWarps = kDecThreads / 32;
 constexpr int kDecQT = 4;          // queries scored together
 constexpr int kDecRows = 4;        // rows a warp has in flight
 
+constexpr int kDecMaxSplits = 64; // thread blocks that may share a head
 constexpr int kDecMaxLayers = 64;  // layers per launch (the pointers travel as a kernel argument)
 
 struct DecodePtrs {                // per-layer device pointers, indexed by layer - layer0
@@ -90,12 +91,21 @@ decode_attend_kernel(DecodePtrs ptrs, int layer0, const int* __restrict__ held, 
 #pragma unroll
       for (int d = 0; d < DPL; ++d) acc[qi][d] = 0.f;
     }
+    // the rows of the next round are requested before the current round is worked on
+    RowFrag<DPL> kn[kDecRows], vn[kDecRows];
+#pragma unroll
+    for (int j = 0; j < kDecRows; ++j) {
+      const int row = r0 + warp + j * kDecWarps;
+      if (row < r1) { kn[j].load(kbase + (size_t)row * D, lane); vn[j].load(vbase + (size_t)row * D, lane); }
+    }
     for (int r = r0 + warp; r < r1; r += kDecWarps * kDecRows) {
       RowFrag<DPL> kf[kDecRows], vf[kDecRows];
 #pragma unroll
+      for (int j = 0; j < kDecRows; ++j) { kf[j] = kn[j]; vf[j] = vn[j]; }
+#pragma unroll
       for (int j = 0; j < kDecRows; ++j) {
-        const int row = r + j * kDecWarps;
-        if (row < r1) { kf[j].load(kbase + (size_t)row * D, lane); vf[j].load(vbase + (size_t)row * D, lane); }
+        const int row = r + kDecWarps * kDecRows + j * kDecWarps;
+        if (row < r1) { kn[j].load(kbase + (size_t)row * D, lane); vn[j].load(vbase + (size_t)row * D, lane); }
       }
       float s[kDecRows][kDecQT];
 #pragma unroll
@@ -172,18 +182,37 @@ decode_attend_kernel(DecodePtrs ptrs, int layer0, const int* __restrict__ held, 
   __threadfence();
   const float* head_scratch = scratch + (size_t)(lz * BH + bh) * splits * GQ * (D + 2);
   float* out = ptrs.out[lz] + (size_t)(b * Hkv + h) * GQ * D;
-  for (int e = tid; e < GQ * D; e += kDecThreads) {
-    const int gq = e / D, d = e % D;
-    float mm = -INFINITY;
-    for (int sp = 0; sp < splits; ++sp) mm = fmaxf(mm, head_scratch[((size_t)sp * GQ + gq) * (D + 2) + D]);
-    float num = 0.f, den = 0.f;
-    for (int sp = 0; sp < splits; ++sp) {
-      const float* pr = head_scratch + ((size_t)sp * GQ + gq) * (D + 2);
-      const float wgt = fast_exp2(pr[D] - mm);
-      num = fmaf(pr[d], wgt, num);
-      den = fmaf(pr[D + 1], wgt, den);
+  float* wgt_s = &part_s[0][0][0];                      // [splits][kDecQT] weights, then [kDecQT] denominators
+  for (int c0 = 0; c0 < GQ; c0 += kDecQT) {
+    __syncthreads();
+    // weight of every split for the chunk's queries: 2^(max of the split - overall max)
+    if (tid < kDecQT * 32) {
+      const int qi = tid >> 5, gq = c0 + qi;
+      float mm = -INFINITY;
+      if (gq < GQ) for (int sp = lane; sp < splits; sp += 32) mm = fmaxf(mm, head_scratch[((size_t)sp * GQ + gq) * (D + 2) + D]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, o));
+      float den = 0.f;
+      if (gq < GQ) for (int sp = lane; sp < splits; sp += 32) {
+        const float* pr = head_scratch + ((size_t)sp * GQ + gq) * (D + 2);
+        const float wgt = fast_exp2(pr[D] - mm);
+        wgt_s[sp * kDecQT + qi] = wgt;
+        den = fmaf(pr[D + 1], wgt, den);
+      }
+      // the denominators are added in a fixed order: lane partial sums, then a butterfly
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xFFFFFFFFu, den, o);
+      if (lane == 0) wgt_s[kDecMaxSplits * kDecQT + qi] = den;
     }
-    out[e] = num / den;
+    __syncthreads();
+    for (int e = tid; e < kDecQT * D; e += kDecThreads) {
+      const int qi = e / D, d = e % D, gq = c0 + qi;
+      if (gq >= GQ) continue;
+      float num = 0.f;
+#pragma unroll 8
+      for (int sp = 0; sp < splits; ++sp) num = fmaf(head_scratch[((size_t)sp * GQ + gq) * (D + 2) + d], wgt_s[sp * kDecQT + qi], num);
+      out[(size_t)gq * D + d] = num / wgt_s[kDecMaxSplits * kDecQT + qi];
+    }
   }
   if (tid == 0) tickets[lz * BH + bh] = 0;
 }

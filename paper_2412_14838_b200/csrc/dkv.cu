@@ -889,8 +889,10 @@ int dkv_decode_attend(dkv_ctx* c, int32_t layer0, int32_t n_layers, int32_t nq, 
   }
   for (int l0 = 0; l0 < n_layers; l0 += kDecMaxLayers) {
     const int nl = n_layers - l0 < kDecMaxLayers ? n_layers - l0 : kDecMaxLayers;
-    // enough thread blocks to fill the GPU a few times over, each with at least a few dozen rows
-    int splits = (4 * c->n_sms + BH * nl - 1) / (BH * nl);
+    // a launch over few heads is latency-bound: one resident wave of thread blocks (two fit an SM); one over many
+    // heads is bandwidth-bound: a few waves, for more loads in flight; every block gets at least a few dozen rows
+    const int waves = BH * nl >= c->n_sms ? 4 : 2;
+    int splits = (waves * c->n_sms + BH * nl - 1) / (BH * nl);
     const int most = (s.rows + 31) / 32;
     if (splits > most) splits = most;
     if (splits > 64) splits = 64;
