@@ -40,11 +40,11 @@ NOMINAL_HBM_GBS = 8000.0
 # the kernel source they were measured on, for that per-layer shape and for four-layer groups only: any other
 # source hash, shape or grouping reports null.
 NCU_TRAFFIC = {
-    "kernel_sha256": "ef8cc89c855a0c39d423e3ff3d2614f1774b61c2594eeadda7494d8e1d00186e",
+    "kernel_sha256": "18ec10036a730195d2c8785c46866764b5bd7c9edc3f1f69259818042292df59",
     "shape": (8, 128, 1, 32768, 32),          # Hkv, D, Bt, S, ws
     "layers_per_launch": 4,
-    "live_bytes_per_launch": 477_236_480 + 5_111_552,
-    "cold_bytes_per_launch": 541_780_000 + 8_060_000,
+    "live_bytes_per_launch": 480_865_280 + 6_463_488,
+    "cold_bytes_per_launch": 541_795_840 + 8_040_704,
 }
 
 
