@@ -157,3 +157,49 @@ def test_pass_scored_from_log_denominators_matches_oracle(name):
         check_properties(g)
     finally:
         g.close()
+
+
+def torch_window_lse(w, q_dev, k_dev):
+    """The window rows' log-denominators as a prefill attention kernel would hand them over (fp32, computed
+    with torch on the device from the same bf16 inputs): an INPUT of the one-sweep pass, not an expected value."""
+    hidden = (torch.arange(w.S, device="cuda")[None, :] > (w.P + torch.arange(w.ws, device="cuda"))[:, None])
+    qf = q_dev.view(torch.bfloat16).float().view(w.Bt, w.Hkv, w.G * w.ws, w.D)
+    kf = k_dev.view(torch.bfloat16).float().view(w.Bt, w.Hkv, w.S, w.D)
+    logits = torch.matmul(qf, kf.transpose(-1, -2)).view(w.Bt, w.Hq, w.ws, w.S) / float(np.sqrt(w.D))
+    return torch.logsumexp(logits.masked_fill(hidden, float("-inf")), dim=-1).contiguous()
+
+
+@pytest.mark.parametrize("name", ["mistral32k", "qwen16k"])
+def test_full_size_one_sweep_pass_sampled(name):
+    """The one-sweep pass at full size, in the launch configuration the benchmark times: sampled heads against the
+    oracle's one-sweep scores for the very lse values the pass was given, and the per-layer counts replayed by the
+    oracle on the pass's own stored scores."""
+    from tests.test_gpu_pass import replay_counts
+    w = synth.WORKLOADS[name]
+    g = GpuPass(w, keep_inputs=False)
+    try:
+        lse = [torch_window_lse(w, g.q[l], g.k[l]) for l in range(w.L)]
+        g.run_with = lambda: B.dkv_run_prefill_pass_lse(g.h, g.q, g.k, g.v, lse, g.kb, g.vb)
+        g.run()
+        check_properties(g)
+        want_counts = replay_counts(g)
+        assert (g.counts == want_counts).all()
+        rng = np.random.default_rng(w.cid + 7)
+        samples = [(int(rng.integers(w.L)), int(rng.integers(w.Bt)), int(rng.integers(w.Hkv))) for _ in range(2)]
+        samples.append((w.L - 1, w.Bt - 1, w.Hkv - 1))
+        near = 0
+        for (l, b, h) in samples:
+            t = synth.layer_inputs(w, l, want_v=False)
+            G = w.G
+            q = synth.bf16_bits_to_f64(t["q"][b:b + 1, h * G:(h + 1) * G])
+            k = synth.bf16_bits_to_f64(t["k"][b:b + 1, h:h + 1])
+            lse_bh = lse[l][b:b + 1, h * G:(h + 1) * G].cpu().numpy().astype(np.float64)
+            ref = O.window_scores_from_lse(q, k, lse_bh, w.ws, w.pool)["score"][0, 0]
+            U.assert_scores_close(g.scores(l)[b, h], ref, f"{name} one-sweep l={l} b={b} h={h}")
+            n = int(want_counts[b, l])
+            idx, _ = g.kept(l)
+            _, ev = U.select_matches(ref, idx[b, h, :n], n)
+            near += ev
+        print(f"[{name}] one-sweep pass: sampled heads ok; near-tie events {near}")
+    finally:
+        g.close()
