@@ -412,7 +412,8 @@ def run_gpu(args, w):
         dt = (time.perf_counter() - t0) / e2e_steps
         dt = max_over_ranks(dt)
         h2d = sum(t.numel() * 2 for t in hq) + sum(t.numel() * 2 for t in hk) + sum(t.numel() * 2 for t in hv)
-        d2h = sum(t.numel() * 2 for t in okb) + sum(t.numel() * 2 for t in ovb) + counts.nbytes
+        # copied back: the counts and the valid rows (count + ws) of every head's K and V buffers
+        d2h = int((counts.astype(np.int64) + w.ws).sum()) * w.Hkv * w.D * 2 * 2 + counts.nbytes
         e2e = {"value": whole_job_value(tokens, world, dt), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                "ms_per_step": dt * 1e3, "steps": e2e_steps, "api": "dkv_run_prefill_pass_host (pinned host buffers)"}
 

@@ -199,7 +199,8 @@ int dkv_run_prefill_pass_lse(dkv_ctx* ctx, const void* const* q_win, const void*
 
 /* The same pass with all tensors in HOST memory (pinned memory recommended): each layer's q, k, v
  * are copied to device staging buffers owned by the context, processed, and after the last update
- * every layer's kb/vb (full fixed-stride buffers) and the counts are copied back.  Synchronises.
+ * the counts and, of every layer's kb/vb, the valid rows of every head (count + ws; the rest of the
+ * fixed-stride host buffers is left untouched) are copied back.  Synchronises.
  * q_win, k, v, kb, vb : host arrays of L HOST pointers; counts_out : host int32 [Bt, L]. */
 int dkv_run_prefill_pass_host(dkv_ctx* ctx, const void* const* q_win, const void* const* k,
                               const void* const* v, void* const* kb, void* const* vb, int32_t* counts_out);

@@ -828,12 +828,23 @@ int dkv_run_prefill_pass_host(dkv_ctx* c, const void* const* q_win, const void* 
       if ((rc = do_shrink(c, 0, l + 1, c->st_kb, c->st_vb, st))) return rc;
     }
   }
-  for (int l = 0; l < s.L; ++l) {
-    DKV_CUDA(c, cudaMemcpyAsync(kb[l], c->st_kb[l], layer_buf_bytes(s), cudaMemcpyDeviceToHost, st));
-    DKV_CUDA(c, cudaMemcpyAsync(vb[l], c->st_vb[l], layer_buf_bytes(s), cudaMemcpyDeviceToHost, st));
-  }
-  if (counts_out)
-    DKV_CUDA(c, cudaMemcpyAsync(counts_out, c->d_count, sizeof(int) * s.Bt * s.L, cudaMemcpyDeviceToHost, st));
+  // The final counts come back first; then only the valid rows of every head (count + ws of the fixed stride)
+  // are copied out, one strided copy per (layer, sample, tensor).
+  std::vector<int> counts((size_t)s.Bt * s.L);
+  DKV_CUDA(c, cudaMemcpyAsync(counts.data(), c->d_count, sizeof(int) * s.Bt * s.L, cudaMemcpyDeviceToHost, st));
+  DKV_CUDA(c, cudaStreamSynchronize(st));
+  const size_t row = (size_t)s.D * 2, head_pitch = (size_t)s.rows * row, sample = (size_t)s.Hkv * head_pitch;
+  for (int l = 0; l < s.L; ++l)
+    for (int b = 0; b < s.Bt; ++b) {
+      const size_t valid = (size_t)(counts[(size_t)b * s.L + l] + s.ws) * row;
+      DKV_CUDA(c, cudaMemcpy2DAsync(static_cast<char*>(kb[l]) + b * sample, head_pitch,
+                                    static_cast<const char*>(c->st_kb[l]) + b * sample, head_pitch, valid, s.Hkv,
+                                    cudaMemcpyDeviceToHost, st));
+      DKV_CUDA(c, cudaMemcpy2DAsync(static_cast<char*>(vb[l]) + b * sample, head_pitch,
+                                    static_cast<const char*>(c->st_vb[l]) + b * sample, head_pitch, valid, s.Hkv,
+                                    cudaMemcpyDeviceToHost, st));
+    }
+  if (counts_out) memcpy(counts_out, counts.data(), sizeof(int) * s.Bt * s.L);
   DKV_CUDA(c, cudaStreamSynchronize(cp));
   DKV_CUDA(c, cudaStreamSynchronize(st));
   return DKV_OK;
