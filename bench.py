@@ -141,8 +141,9 @@ def workload_config(w):
     return {"workload": w.name, "layers": w.L, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D, "batch": w.Bt,
             "prefix_len": w.S, "window": w.ws, "pool": w.pool, "avg_budget": w.N, "layer_max": w.Bl,
             "update_interval": w.m, "recipe": w.recipe, "seed": synth.BASE_SEED,
-            "l2": "inputs (K+V of all layers, %.1f GB) exceed L2; no flush needed" %
-                  (2 * w.L * w.k_bytes_per_layer() / 1e9)}
+            "l2": ("inputs (K+V of all layers, %.2f GB) exceed L2; no flush needed" if 2 * w.L * w.k_bytes_per_layer() > 256e6
+                   else "inputs (K+V of all layers, %.2f GB) fit L2 and are NOT flushed between steps: a parity-size "
+                        "workload, not a bench line") % (2 * w.L * w.k_bytes_per_layer() / 1e9)}
 
 
 # ------------------------------------------------------------------------------------ clocks
