@@ -96,23 +96,24 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after `limit` clock ticks, records the failure (status[0] = the first wait site that
+// Bounded wait: true once the barrier's phase is complete; gives up after `limit` clock ticks (false), records the failure (status[0] = the first wait site that
 // gave up, status[2] = its CTA) and lets the kernel run to its end: once the CTA's abort flag is up no wait
 // blocks, no further copy or MMA is issued, and the CTA drains what it has in flight before it frees its
 // tensor memory.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
                                           long long limit) {
-  if (*abort_flag) return;
-  if (mbar_try(bar, parity)) return;
+  if (mbar_try(bar, parity)) return true;      // the usual case costs one instruction: the control threads share
+  if (*abort_flag) return false;               // their schedulers with the softmax warps and every instruction waits its turn
   const long long t0 = clock64();
   while (!mbar_try(bar, parity)) {
-    if (*abort_flag) return;
+    if (*abort_flag) return false;
     if (clock64() - t0 > limit) {
       *abort_flag = 1;
       if (atomicCAS(status, 0, code) == 0) status[2] = (int)blockIdx.x;
-      return;
+      return false;
     }
   }
+  return true;
 }
 // After an abort: wait a short while for something of this CTA's own that is still in flight.  Never records.
 __device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
@@ -136,7 +137,27 @@ __device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// A operand from tensor memory (128 rows = lanes, 16-bit elements packed two per column), B from shared memory.
+// The eight k-steps of a 128-dim tile issued as one block: the descriptors of the steps differ in their low words
+// only (32 bytes = 2 units per step inside a 64-column half, A_HALF / B_HALF units to the second half), so the
+// issuing thread spends two additions per MMA instead of rebuilding two 64-bit descriptors.
+template <int A_HALF, int B_HALF>
+__device__ __forceinline__ void tc_mma_x8(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc) {
+#define DKV_MMA_STEP(OFF, P)                                                                             \
+      "add.u32 la, %1, " OFF ";\n\tadd.u32 lb, %2, " OFF ";\n\tmov.b64 da, {la, %3};\n\tmov.b64 db, {lb, %3};\n\t" \
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, " P ";\n\t"
+#define DKV_MMA_STEP2(OFF, P)                                                                            \
+      "add.u32 la, %1, %5;\n\tadd.u32 la, la, " OFF ";\n\tadd.u32 lb, %2, %6;\n\tadd.u32 lb, lb, " OFF ";\n\t"    \
+      "mov.b64 da, {la, %3};\n\tmov.b64 db, {lb, %3};\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, " P ";\n\t"
+  asm volatile(
+      "{\n\t.reg .pred pf, pt;\n\t.reg .b64 da, db;\n\t.reg .b32 la, lb;\n\t"
+      "setp.ne.b32 pf, 0, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+      DKV_MMA_STEP("0", "pf") DKV_MMA_STEP("2", "pt") DKV_MMA_STEP("4", "pt") DKV_MMA_STEP("6", "pt")
+      DKV_MMA_STEP2("0", "pt") DKV_MMA_STEP2("2", "pt") DKV_MMA_STEP2("4", "pt") DKV_MMA_STEP2("6", "pt")
+      "}"
+      ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "n"(A_HALF), "n"(B_HALF) : "memory");
+#undef DKV_MMA_STEP
+#undef DKV_MMA_STEP2
+}
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
   uint32_t r[16];
   asm volatile(
@@ -290,9 +311,9 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int tile = 0, nq = 0;
-      int last_on[kStages];                    // last tile whose copy went to each ring stage (-1: none)
-      for (int s = 0; s < kStages; ++s) last_on[s] = -1;
-      for (int jb = 0; jb < 2; ++jb) {
+      int withheld = -1;                       // the tile (counted over the launch) whose copy the test hook skipped
+      bool ok = true;                          // false once a wait has run out, here or in another thread
+      for (int jb = 0; jb < 2 && ok; ++jb) {
         const Params& p = jb ? job1 : job0;
         if (p.mode == kNone) continue;
         const Maps& maps = jb ? maps1 : maps0;
@@ -302,15 +323,15 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
         SegIter it(p, blockIdx.x, gridDim.x);
         Seg sg;
         int job_tile = 0;
-        while (it.next(sg)) {
+        while (ok && it.next(sg)) {
           const int hh = sg.bh % p.hpl;
           const CUtensorMap* q_map = &maps.q[sg.bh / p.hpl];
           const CUtensorMap* k_map = &maps.k[sg.bh / p.hpl];
           if (sg.new_head) {
             // every MMA that read the previous queries must have finished: the last tile of either issuer
             for (int last = tile - 1; last >= 0 && last >= tile - 2; --last)
-              mbar_wait(EMPTY(last % kStages), (last / kStages) & 1, abort_flag, p.status, 101, p.wait_cycles);
-            if (!*abort_flag) {
+              ok = ok && mbar_wait(EMPTY(last % kStages), (last / kStages) & 1, abort_flag, p.status, 101, p.wait_cycles);
+            if (ok) {
               mbar_expect_tx(QFULL, (uint32_t)(p.nmblk * halves) * kHalfBytes);
               for (int h = 0; h < halves; ++h)
                 for (int mb = 0; mb < p.nmblk; ++mb)
@@ -320,22 +341,22 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
           }
           for (int i = 0; i < sg.ntiles; ++i, ++tile, ++job_tile) {
             const int s = tile % kStages, n = tile / kStages;
-            mbar_wait(EMPTY(s), (n & 1) ^ 1, abort_flag, p.status, 102, p.wait_cycles);
-            if (*abort_flag) break;
-            if (job_tile == withhold) continue;          // test hook: this tile never arrives
+            if (!mbar_wait(EMPTY(s), (n & 1) ^ 1, abort_flag, p.status, 102, p.wait_cycles)) { ok = false; break; }
+            if (job_tile == withhold) { withheld = tile; continue; }   // test hook: this tile never arrives
             mbar_expect_tx(FULL(s), tile_bytes);
             for (int h = 0; h < halves; ++h)
               tma_load_3d(smem_u32(k_smem + (s * 2 + h) * kHalfBytes), k_map, FULL(s), 64 * h, sg.key0 + i * kTileKeys, hh);
-            last_on[s] = tile;
           }
-          if (*abort_flag) break;
         }
-        if (*abort_flag) break;
       }
-      if (*abort_flag) {
-        // copies of this CTA that may still be on their way must land before its shared memory is given up
-        for (int s = 0; s < kStages; ++s)
-          if (last_on[s] >= 0) mbar_drain(FULL(s), (last_on[s] / kStages) & 1);
+      if (!ok || *abort_flag) {
+        // copies of this CTA that may still be on their way must land before its shared memory is given up:
+        // for every ring stage, the last tile (below `tile`) whose copy went there
+        for (int s = 0; s < kStages; ++s) {
+          int last = tile - 1 - ((tile - 1 - s) % kStages + kStages) % kStages;
+          if (last == withheld) last -= kStages;
+          if (last >= 0) mbar_drain(FULL(s), (last / kStages) & 1);
+        }
         if (nq > 0) mbar_drain(QFULL, (nq - 1) & 1);
       }
     }
@@ -346,6 +367,8 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
     // tensor core needs to run them.
     if (lane == 0) {
       const int which = warp == 1 ? 0 : 1;
+      const uint64_t kdesc0 = smem_desc(smem_u32(k_smem)), qdesc0 = smem_desc(smem_u32(q_smem));
+      const uint32_t kq_lo[2] = {(uint32_t)kdesc0, (uint32_t)qdesc0}, desc_hi = (uint32_t)(kdesc0 >> 32);
       int tile = 0, nq = 0;
       bool q_wait = false;
       for (int jb = 0; jb < 2; ++jb) {
@@ -360,17 +383,28 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
           if (sg.new_head) { q_wait = true; ++nq; }
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
             if ((tile & 1) != which) continue;
+            bool ok = true;
             if (q_wait) {
               q_wait = false;
-              mbar_wait(QFULL, (nq - 1) & 1, abort_flag, p.status, 103, p.wait_cycles);
+              ok = mbar_wait(QFULL, (nq - 1) & 1, abort_flag, p.status, 103, p.wait_cycles);
             }
             const int s = tile % kStages, n = tile / kStages, t = tile & tmask, nt = tile >> tshift;
-            mbar_wait(FULL(s), n & 1, abort_flag, p.status, 104, p.wait_cycles);
-            mbar_wait(TEMPTY(t), (nt & 1) ^ 1, abort_flag, p.status, 105, p.wait_cycles);
-            if (*abort_flag) continue;                   // nothing more is issued once a wait has run out
+            ok = ok && mbar_wait(FULL(s), n & 1, abort_flag, p.status, 104, p.wait_cycles);
+            ok = ok && mbar_wait(TEMPTY(t), (nt & 1) ^ 1, abort_flag, p.status, 105, p.wait_cycles);
+            if (!ok) continue;                           // nothing more is issued once a wait has run out
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(t * scols);
-            if (p.mode == kStats) {
+            if (ksteps == 8) {
+              // low descriptor words: the tile's ring stage, the queries' row block; 16-byte units
+              const uint32_t k_lo = kq_lo[0] + ((uint32_t)(s * 2 * kHalfBytes) >> 4);
+              if (p.mode == kStats) {
+                for (int mb = 0; mb < p.nmblk; ++mb)
+                  tc_mma_x8<((2 * kHalfBytes) >> 4), (kHalfBytes >> 4)>(d_tmem + mb * 128, kq_lo[1] + ((uint32_t)(mb * kHalfBytes) >> 4),
+                                                                     k_lo, desc_hi, p.idesc);
+              } else {
+                tc_mma_x8<(kHalfBytes >> 4), ((2 * kHalfBytes) >> 4)>(d_tmem, k_lo, kq_lo[1], desc_hi, p.idesc);
+              }
+            } else if (p.mode == kStats) {
               for (int mb = 0; mb < p.nmblk; ++mb)
                 for (int ks = 0; ks < ksteps; ++ks) {
                   const uint64_t a = smem_desc(smem_u32(q_smem + (ks >> 2) * (2 * kHalfBytes) + mb * kHalfBytes) + (ks & 3) * 32);
