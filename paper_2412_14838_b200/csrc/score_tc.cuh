@@ -186,6 +186,30 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
+// Packed fp32 pairs (one instruction for two lanes of arithmetic): the softmax warps' instruction count is what
+// the single-thread producer and issuers compete with for issue slots.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+// (s.x, s.y) += (2^(x0 * scale + c0), 2^(x1 * scale + c1))
+__device__ __forceinline__ uint64_t exp2_acc2(uint64_t sum, float x0, float x1, uint64_t scale, uint64_t c) {
+  float t0, t1;
+  unpack2(fma2(pack2(x0, x1), scale, c), t0, t1);
+  return add2(sum, pack2(fast_exp2(t0), fast_exp2(t1)));
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory operand descriptor: K-major, 128-byte swizzle, rows 128 B apart, 8-row groups 1024 B apart.
@@ -272,9 +296,9 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* q_smem = smem;                              // [half][256 rows][128 B]
   uint8_t* k_smem = smem + kQRegion;                   // [stage][half][128 rows][128 B]
-  float* lse_s = reinterpret_cast<float*>(k_smem + kKRegion);          // [256] lse2 per window row (sweep 2)
-  float2* merge_s = reinterpret_cast<float2*>(lse_s + 256);            // [3][256] partials of column parts 1..3 (sweep 1)
-  float* raw_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(lse_s) + kMiscBytes);   // [half][kMaxSegTiles * 128]
+  float* nlse_s = reinterpret_cast<float*>(k_smem + kKRegion);         // [256] minus lse2 per window row (sweep 2)
+  float2* merge_s = reinterpret_cast<float2*>(nlse_s + 256);            // [3][256] partials of column parts 1..3 (sweep 1)
+  float* raw_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(nlse_s) + kMiscBytes);   // [half][kMaxSegTiles * 128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(raw_s) + kRawBytes);
   // barriers: full[kStages], empty[kStages], tmem_full[4], tmem_empty[4], q_full, drain[2]
   __shared__ uint32_t tmem_base_s;
@@ -444,6 +468,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
       SegIter it(p, blockIdx.x, gridDim.x);
       Seg sg;
       const int tmask = p.nmblk == 1 ? 3 : 1, tshift = p.nmblk == 1 ? 2 : 1, scols = p.nmblk == 1 ? 128 : 256;
+      const uint64_t scale22 = pack2(p.scale2, p.scale2);
       while (it.next(sg)) {
         if (p.mode == kStats) {
           // ------------------------------------------------------------ sweep 1: (max, sum) per window row
@@ -483,15 +508,15 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
                 if (cm == -INFINITY) continue;
                 const float mnew = fmaxf(mx[mb], cm * p.scale2);
                 if (mnew > mx[mb]) { sum[mb] *= fast_exp2(mx[mb] - mnew); mx[mb] = mnew; }
-                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-                const float neg = -mx[mb];
+                uint64_t s01 = 0ull, s23 = 0ull;            // four partial sums, as two packed pairs
+                const uint64_t neg2 = pack2(-mx[mb], -mx[mb]);
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
-                  s0 += fast_exp2(fmaf(xv[e], p.scale2, neg));
-                  s1 += fast_exp2(fmaf(xv[e + 1], p.scale2, neg));
-                  s2 += fast_exp2(fmaf(xv[e + 2], p.scale2, neg));
-                  s3 += fast_exp2(fmaf(xv[e + 3], p.scale2, neg));
+                  s01 = exp2_acc2(s01, xv[e], xv[e + 1], scale22, neg2);
+                  s23 = exp2_acc2(s23, xv[e + 2], xv[e + 3], scale22, neg2);
                 }
+                float s0, s1, s2, s3;
+                unpack2(s01, s0, s1); unpack2(s23, s2, s3);
                 sum[mb] += (s0 + s1) + (s2 + s3);
               }
             }
@@ -545,7 +570,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
               }
               lse = m + log2f(l);
             }
-            lse_s[sid] = lse;
+            nlse_s[sid] = -lse;
           }
           asm volatile("bar.sync 1, 512;" ::: "memory");
           const int nchunk = p.nq16 >> 4;               // 16-column chunks; this warp takes half, half+2, ...
@@ -556,7 +581,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
             mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 107, p.wait_cycles);
             tc_fence_after();
             const uint32_t taddr = lane_addr + (uint32_t)(t * scols);
-            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            uint64_t a01 = 0ull, a23 = 0ull;               // four partial sums, as two packed pairs
             if (half >= nchunk) {                              // a single chunk (ws*G <= 16): nothing for this warp to read
               tc_fence_before();
               __syncwarp();
@@ -577,23 +602,21 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
               }
 #pragma unroll
               for (int e = 0; e < 16; e += 4) {
-                const float4 ls = *reinterpret_cast<const float4*>(&lse_s[c0 * 16 + e]);
-                a0 += fast_exp2(fmaf(x0[e], p.scale2, -ls.x));
-                a1 += fast_exp2(fmaf(x0[e + 1], p.scale2, -ls.y));
-                a2 += fast_exp2(fmaf(x0[e + 2], p.scale2, -ls.z));
-                a3 += fast_exp2(fmaf(x0[e + 3], p.scale2, -ls.w));
+                const ulonglong2 ls = *reinterpret_cast<const ulonglong2*>(&nlse_s[c0 * 16 + e]);   // minus lse, four rows
+                a01 = exp2_acc2(a01, x0[e], x0[e + 1], scale22, ls.x);
+                a23 = exp2_acc2(a23, x0[e + 2], x0[e + 3], scale22, ls.y);
               }
               if (c1 < nchunk) {
 #pragma unroll
                 for (int e = 0; e < 16; e += 4) {
-                  const float4 ls = *reinterpret_cast<const float4*>(&lse_s[c1 * 16 + e]);
-                  a0 += fast_exp2(fmaf(x1[e], p.scale2, -ls.x));
-                  a1 += fast_exp2(fmaf(x1[e + 1], p.scale2, -ls.y));
-                  a2 += fast_exp2(fmaf(x1[e + 2], p.scale2, -ls.z));
-                  a3 += fast_exp2(fmaf(x1[e + 3], p.scale2, -ls.w));
+                  const ulonglong2 ls = *reinterpret_cast<const ulonglong2*>(&nlse_s[c1 * 16 + e]);
+                  a01 = exp2_acc2(a01, x1[e], x1[e + 1], scale22, ls.x);
+                  a23 = exp2_acc2(a23, x1[e + 2], x1[e + 3], scale22, ls.y);
                 }
               }
             }
+            float a0, a1, a2, a3;
+            unpack2(a01, a0, a1); unpack2(a23, a2, a3);
             my_raw[i * kTileKeys + row] = (a0 + a1) + (a2 + a3);
           }
           asm volatile("bar.sync 1, 512;" ::: "memory");
