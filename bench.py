@@ -40,11 +40,11 @@ NOMINAL_HBM_GBS = 8000.0
 # the kernel source they were measured on, for that per-layer shape and for four-layer groups only: any other
 # source hash, shape or grouping reports null.
 NCU_TRAFFIC = {
-    "kernel_sha256": "18ec10036a730195d2c8785c46866764b5bd7c9edc3f1f69259818042292df59",
+    "kernel_sha256": "fbec4372a65a013bb9bac9081330579d55d3ffdec06bbf7f90f1e9fc13110969",
     "shape": (8, 128, 1, 32768, 32),          # Hkv, D, Bt, S, ws
     "layers_per_launch": 4,
-    "live_bytes_per_launch": 480_865_280 + 6_463_488,
-    "cold_bytes_per_launch": 541_795_840 + 8_040_704,
+    "live_bytes_per_launch": 479_409_664 + 5_171_968,
+    "cold_bytes_per_launch": 541877248 + 7847424,
 }
 
 
