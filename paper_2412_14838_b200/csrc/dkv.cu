@@ -240,6 +240,14 @@ bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, con
   return true;
 }
 
+// The scoring kernel for two jobs (either may be kNone): the specialised build when every job has exactly 128 window
+// rows of 128 dims, the general one otherwise.
+void launch_tc(int grid, cudaStream_t st, const tc::Maps& m0, const tc::Maps& m1, const tc::Params& j0, const tc::Params& j1) {
+  auto fast = [](const tc::Params& p) { return p.mode == tc::kNone || (p.M == 128 && p.D == 128); };
+  if (fast(j0) && fast(j1)) tc::score_tc_kernel<true><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(m0, m1, j0, j1);
+  else tc::score_tc_kernel<false><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(m0, m1, j0, j1);
+}
+
 // One launch: sweep 2 of the `en` layers from `emit_layer` (if >= 0), then sweep 1 of the `sn` layers from
 // `stats_layer` (if >= 0).  In the pass the emit layers are the ones the previous launch streamed.  `sbuf`, `ebuf`: statistics scratch of either job.
 int launch_score(dkv_ctx* c, int stats_layer, int sn, const void* const* sq, const void* const* sk, int sbuf,
@@ -253,7 +261,7 @@ int launch_score(dkv_ctx* c, int stats_layer, int sn, const void* const* sq, con
   if (emit_layer >= 0 && !make_job(c, tc::kEmit, emit_layer, en, eq, ek, scores_out, ebuf, &m0, &j0, emit_lse)) return DKV_ERR_CUDA;
   if (stats_layer >= 0 && !make_job(c, tc::kStats, stats_layer, sn, sq, sk, nullptr, sbuf, &m1, &j1)) return DKV_ERR_CUDA;
   ProfScope ps(c, stats_layer >= 0 ? DKV_STEP_SCORE_STATS : DKV_STEP_SCORE_EMIT, 1, st);
-  tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(m0, m1, j0, j1);
+  launch_tc(c->tc_grid, st, m0, m1, j0, j1);
   DKV_LAUNCHED(c);
   return DKV_OK;
 }
@@ -267,7 +275,7 @@ int do_score_lse(dkv_ctx* c, int layer, const void* q, const void* k, const floa
   none.mode = tc::kNone;
   if (!make_job(c, tc::kEmit, layer, 1, &q, &k, scores_out, layer % 3, &maps, &job, &lse)) return DKV_ERR_CUDA;
   ProfScope ps(c, DKV_STEP_SCORE_EMIT, 1, st);
-  tc::score_tc_kernel<<<c->tc_grid, tc::kThreads, tc::kSmemBytes, st>>>(maps, maps, job, none);
+  launch_tc(c->tc_grid, st, maps, maps, job, none);
   DKV_LAUNCHED(c);
   c->scored[layer] = 1;
   c->selected[layer] = c->gathered[layer] = c->stale[layer] = 0;
@@ -598,7 +606,8 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
   TRY(cudaMalloc(&c->d_cand, sizeof(uint2) * s.L * layer_scores(s)));
   TRY(cudaMalloc(&c->d_cand_n, sizeof(unsigned int) * s.Bt));
   TRY(cudaMalloc(&c->d_tc_stats, sizeof(float2) * 3 * tc::kMaxGroup * heads * c->tc_slots * 256));
-  TRY(cudaFuncSetAttribute(tc::score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  TRY(cudaFuncSetAttribute(tc::score_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  TRY(cudaFuncSetAttribute(tc::score_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   for (int i = 0; i < kSideStreams; ++i) TRY(cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking));
   TRY(cudaStreamCreateWithFlags(&c->gstream, cudaStreamNonBlocking));
   TRY(cudaEventCreateWithFlags(&c->ev_gfork, cudaEventDisableTiming));
@@ -993,8 +1002,10 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
       if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return DKV_ERR_CUDA;
       int sms = 0;
       if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return DKV_ERR_CUDA;
-      if (cudaFuncSetAttribute(tc::score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes) !=
-          cudaSuccess)
+      if (cudaFuncSetAttribute(tc::score_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes) !=
+              cudaSuccess ||
+          cudaFuncSetAttribute(tc::score_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes) !=
+              cudaSuccess)
         return DKV_ERR_CUDA;
       g.ptr = static_cast<unsigned char*>(ptr);
       g.sms = sms;
@@ -1040,11 +1051,11 @@ int dkv_score_static(const dkv_config* cfg, const void* q_win, const void* k, fl
   p.stats_grid = grid;
   p.mode = tc::kStats;
   p.idesc = make_idesc(128, 128);
-  tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(maps, maps, p, none);
+  launch_tc(grid, st, maps, maps, p, none);
   if (cudaGetLastError() != cudaSuccess) return DKV_ERR_CUDA;
   p.mode = tc::kEmit;
   p.idesc = make_idesc(128, p.nq16);
-  tc::score_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, st>>>(maps, maps, none, p);
+  launch_tc(grid, st, maps, maps, none, p);
   if (cudaGetLastError() != cudaSuccess) return DKV_ERR_CUDA;
   return DKV_OK;
 }

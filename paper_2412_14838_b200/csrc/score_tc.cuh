@@ -289,6 +289,9 @@ __host__ __device__ __forceinline__ int tile_owner(long long x, long long total,
 
 // ------------------------------------------------------------------------------------------ kernel
 // job0 uses maps0, job1 uses maps1; a job with mode kNone is skipped.
+// kFast: both jobs have exactly 128 window rows of 128 dims (ws*G = 128, D = 128, the shape of the 32/8-head models):
+// the row-block count, the chunk count and the k-step count are then compile-time constants.
+template <bool kFast>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps maps1,
                 const __grid_constant__ Params job0, const __grid_constant__ Params job1) {
@@ -313,6 +316,8 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &abort_s;
+  auto NMBLK = [](const Params& p) { return kFast ? 1 : p.nmblk; };
+  auto DIMS = [](const Params& p) { return kFast ? 128 : p.D; };
 
   if (threadIdx.x == 0) {
     abort_s = 0;
@@ -341,7 +346,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
         const Params& p = jb ? job1 : job0;
         if (p.mode == kNone) continue;
         const Maps& maps = jb ? maps1 : maps0;
-        const int halves = p.D / 64;
+        const int halves = DIMS(p) / 64;
         const uint32_t tile_bytes = (uint32_t)halves * kHalfBytes;
         const int withhold = blockIdx.x == 0 ? p.withhold_tile : -1;
         SegIter it(p, blockIdx.x, gridDim.x);
@@ -356,9 +361,9 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
             for (int last = tile - 1; last >= 0 && last >= tile - 2; --last)
               ok = ok && mbar_wait(EMPTY(last % kStages), (last / kStages) & 1, abort_flag, p.status, 101, p.wait_cycles);
             if (ok) {
-              mbar_expect_tx(QFULL, (uint32_t)(p.nmblk * halves) * kHalfBytes);
+              mbar_expect_tx(QFULL, (uint32_t)(NMBLK(p) * halves) * kHalfBytes);
               for (int h = 0; h < halves; ++h)
-                for (int mb = 0; mb < p.nmblk; ++mb)
+                for (int mb = 0; mb < NMBLK(p); ++mb)
                   tma_load_3d(smem_u32(q_smem + h * (2 * kHalfBytes) + mb * kHalfBytes), q_map, QFULL, 64 * h, 128 * mb, hh);
               ++nq;
             }
@@ -398,8 +403,8 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
       for (int jb = 0; jb < 2; ++jb) {
         const Params& p = jb ? job1 : job0;
         if (p.mode == kNone) continue;
-        const int ksteps = p.D / 16;
-        const int tmask = p.nmblk == 1 ? 3 : 1, tshift = p.nmblk == 1 ? 2 : 1, scols = p.nmblk == 1 ? 128 : 256;
+        const int ksteps = DIMS(p) / 16;
+        const int tmask = NMBLK(p) == 1 ? 3 : 1, tshift = NMBLK(p) == 1 ? 2 : 1, scols = NMBLK(p) == 1 ? 128 : 256;
         SegIter it(p, blockIdx.x, gridDim.x);
         Seg sg;
         while (it.next(sg)) {
@@ -422,14 +427,14 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
               // low descriptor words: the tile's ring stage, the queries' row block; 16-byte units
               const uint32_t k_lo = kq_lo[0] + ((uint32_t)(s * 2 * kHalfBytes) >> 4);
               if (p.mode == kStats) {
-                for (int mb = 0; mb < p.nmblk; ++mb)
+                for (int mb = 0; mb < NMBLK(p); ++mb)
                   tc_mma_x8<((2 * kHalfBytes) >> 4), (kHalfBytes >> 4)>(d_tmem + mb * 128, kq_lo[1] + ((uint32_t)(mb * kHalfBytes) >> 4),
                                                                      k_lo, desc_hi, p.idesc);
               } else {
                 tc_mma_x8<(kHalfBytes >> 4), ((2 * kHalfBytes) >> 4)>(d_tmem, k_lo, kq_lo[1], desc_hi, p.idesc);
               }
             } else if (p.mode == kStats) {
-              for (int mb = 0; mb < p.nmblk; ++mb)
+              for (int mb = 0; mb < NMBLK(p); ++mb)
                 for (int ks = 0; ks < ksteps; ++ks) {
                   const uint64_t a = smem_desc(smem_u32(q_smem + (ks >> 2) * (2 * kHalfBytes) + mb * kHalfBytes) + (ks & 3) * 32);
                   const uint64_t b = smem_desc(smem_u32(k_smem + (s * 2 + (ks >> 2)) * kHalfBytes) + (ks & 3) * 32);
@@ -467,7 +472,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
       if (p.mode == kNone) continue;
       SegIter it(p, blockIdx.x, gridDim.x);
       Seg sg;
-      const int tmask = p.nmblk == 1 ? 3 : 1, tshift = p.nmblk == 1 ? 2 : 1, scols = p.nmblk == 1 ? 128 : 256;
+      const int tmask = NMBLK(p) == 1 ? 3 : 1, tshift = NMBLK(p) == 1 ? 2 : 1, scols = NMBLK(p) == 1 ? 128 : 256;
       const uint64_t scale22 = pack2(p.scale2, p.scale2);
       while (it.next(sg)) {
         if (p.mode == kStats) {
@@ -484,13 +489,13 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
             const bool need_mask = kb0 + 63 > p.P;
 #pragma unroll
             for (int mb = 0; mb < 2; ++mb) {
-              if (mb >= p.nmblk) break;
+              if (mb >= NMBLK(p)) break;
 #pragma unroll
               for (int hh = 0; hh < 2; ++hh) {
                 float xv[32];
                 tc_ld32(taddr + mb * 128 + hh * 32, xv);
                 tc_wait_ld();
-                if (mb + 1 == p.nmblk && hh == 1) {              // last read of this stage: release it
+                if (mb + 1 == NMBLK(p) && hh == 1) {              // last read of this stage: release it
                   tc_fence_before();
                   __syncwarp();
                   if (lane == 0) mbar_arrive(TEMPTY(t));
@@ -533,7 +538,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
 #pragma unroll
             for (int mb = 0; mb < 2; ++mb) {
               const int r = row + 128 * mb;
-              if (mb < p.nmblk && r < p.M) {
+              if (mb < NMBLK(p) && r < p.M) {
                 float m = mx[mb];
 #pragma unroll
                 for (int q = 0; q < 3; ++q) m = fmaxf(m, merge_s[q * 256 + r].x);
@@ -573,7 +578,7 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
             nlse_s[sid] = -lse;
           }
           asm volatile("bar.sync 1, 512;" ::: "memory");
-          const int nchunk = p.nq16 >> 4;               // 16-column chunks; this warp takes half, half+2, ...
+          const int nchunk = kFast ? 8 : p.nq16 >> 4;               // 16-column chunks; this warp takes half, half+2, ...
           float* my_raw = raw_s + half * (kMaxSegTiles * kTileKeys);
           for (int i = 0; i < sg.ntiles; ++i, ++tile) {
             if ((tile & 1) != grp) continue;                   // the other group's tile
