@@ -410,8 +410,11 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
         while (it.next(sg)) {
           // the wait for a head's queries is taken at this issuer's first tile of the head (it may have none)
           if (sg.new_head) { q_wait = true; ++nq; }
-          for (int i = 0; i < sg.ntiles; ++i, ++tile) {
-            if ((tile & 1) != which) continue;
+          // this thread's tiles only: every other one, by the parity of the tile's number over the launch
+          const int tile0 = tile;
+          tile += sg.ntiles;
+          for (int i = (which ^ tile0) & 1, tile_ = tile0 + i; i < sg.ntiles; i += 2, tile_ += 2) {
+            const int tile = tile_;
             bool ok = true;
             if (q_wait) {
               q_wait = false;
@@ -479,8 +482,11 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
           // ------------------------------------------------------------ sweep 1: (max, sum) per window row
           float mx[2] = {-INFINITY, -INFINITY}, sum[2] = {0.f, 0.f};
           const int limit0 = p.P + (row % p.ws), limit1 = p.P + ((row + 128) % p.ws);
-          for (int i = 0; i < sg.ntiles; ++i, ++tile) {
-            if ((tile & 1) != grp) continue;                   // the other group's tile
+          // this thread's tiles only: every other one, by the parity of the tile's number over the launch
+          const int tile0 = tile;
+          tile += sg.ntiles;
+          for (int i = (grp ^ tile0) & 1, tile_ = tile0 + i; i < sg.ntiles; i += 2, tile_ += 2) {
+            const int tile = tile_;
             const int t = tile & tmask, nt = tile >> tshift;
             mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 106, p.wait_cycles);
             tc_fence_after();
@@ -580,8 +586,11 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
           asm volatile("bar.sync 1, 512;" ::: "memory");
           const int nchunk = kFast ? 8 : p.nq16 >> 4;               // 16-column chunks; this warp takes half, half+2, ...
           float* my_raw = raw_s + half * (kMaxSegTiles * kTileKeys);
-          for (int i = 0; i < sg.ntiles; ++i, ++tile) {
-            if ((tile & 1) != grp) continue;                   // the other group's tile
+          // this thread's tiles only: every other one, by the parity of the tile's number over the launch
+          const int tile0 = tile;
+          tile += sg.ntiles;
+          for (int i = (grp ^ tile0) & 1, tile_ = tile0 + i; i < sg.ntiles; i += 2, tile_ += 2) {
+            const int tile = tile_;
             const int t = tile & tmask, nt = tile >> tshift;
             mbar_wait(TFULL(t), nt & 1, abort_flag, p.status, 107, p.wait_cycles);
             tc_fence_after();
