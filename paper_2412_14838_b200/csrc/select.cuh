@@ -85,15 +85,53 @@ __device__ __forceinline__ unsigned int agg_bump(unsigned int* counters, unsigne
   return base + (unsigned int)__popc(peers & ((1u << lane) - 1u));
 }
 
+// One compare-exchange step of a bitonic network on the 64 keys a warp holds in registers: lane j has
+// a = key[base + j] and b = key[base + 32 + j].  `s` is the stride (32, 16, ..., 1), `size` the length of the
+// bitonic sequences being merged; a block of `size` keys is sorted ascending if its first index has bit `size` clear.
+__device__ __forceinline__ void bitonic_step64(unsigned long long& a, unsigned long long& b, int base, int lane, int s, int size) {
+  if (s == 32) {
+    const bool up = ((base + lane) & size) == 0;
+    if ((a > b) == up) { const unsigned long long t = a; a = b; b = t; }
+  } else {
+    const unsigned long long pa = __shfl_xor_sync(0xFFFFFFFFu, a, s), pb = __shfl_xor_sync(0xFFFFFFFFu, b, s);
+    const bool lower = (lane & s) == 0;                       // this lane holds the lower index of its pair
+    const bool up_a = ((base + lane) & size) == 0, up_b = ((base + 32 + lane) & size) == 0;
+    a = (lower == up_a) ? (a < pa ? a : pa) : (a > pa ? a : pa);
+    b = (lower == up_b) ? (b < pb ? b : pb) : (b > pb ? b : pb);
+  }
+}
+
 // Bitonic sort of keys[0 .. sort_n) ascending; sort_n a power of two >= 2.  Strides of 64 and more are
-// done by the whole block with a barrier per stage; the strides below that stay inside 64-key blocks,
-// each owned by one warp, and only need warp barriers.  Ends with a block barrier.
+// done by the whole block in shared memory with a barrier per stage; the strides below that stay inside
+// 64-key blocks, each owned by one warp, which holds its block in registers (two keys per lane) and
+// exchanges by shuffles; the first six merge lengths (2 .. 64) run entirely in registers.  Arrays of
+// fewer than 64 keys use shared memory throughout.  Ends with a block barrier.
 __device__ __forceinline__ void bitonic_sort(unsigned long long* keys, int sort_n) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  const int blk = sort_n < 64 ? sort_n : 64;               // keys per warp-owned block
-  for (int size = 2; size <= sort_n; size <<= 1) {
-    int stride = size >> 1;
-    for (; stride >= 64; stride >>= 1) {
+  if (sort_n < 64) {
+    for (int size = 2; size <= sort_n; size <<= 1) {
+      for (int s = size >> 1; s > 0; s >>= 1) {
+        for (int t = threadIdx.x; t < (sort_n >> 1); t += blockDim.x) {
+          const int lo = ((t & ~(s - 1)) << 1) | (t & (s - 1)), hi = lo + s;
+          const bool up = ((lo & size) == 0);
+          const unsigned long long a = keys[lo], b = keys[hi];
+          if ((a > b) == up) { keys[lo] = b; keys[hi] = a; }
+        }
+        __syncthreads();
+      }
+    }
+    return;
+  }
+  __syncthreads();
+  for (int base = warp * 64; base < sort_n; base += nwarps * 64) {      // merge lengths 2 .. 64 in registers
+    unsigned long long a = keys[base + lane], b = keys[base + 32 + lane];
+    for (int size = 2; size <= 64; size <<= 1)
+      for (int s = size >> 1; s > 0; s >>= 1) bitonic_step64(a, b, base, lane, s, size);
+    keys[base + lane] = a; keys[base + 32 + lane] = b;
+  }
+  __syncthreads();
+  for (int size = 128; size <= sort_n; size <<= 1) {
+    for (int stride = size >> 1; stride >= 64; stride >>= 1) {
       for (int t = threadIdx.x; t < (sort_n >> 1); t += blockDim.x) {
         const int lo = ((t & ~(stride - 1)) << 1) | (t & (stride - 1));
         const int hi = lo + stride;
@@ -103,17 +141,11 @@ __device__ __forceinline__ void bitonic_sort(unsigned long long* keys, int sort_
       }
       __syncthreads();
     }
-    for (int base = warp * blk; base < sort_n; base += nwarps * blk) {
-      for (int s = stride; s > 0; s >>= 1) {
-        if (lane < (blk >> 1)) {
-          const int lo = base + (((lane & ~(s - 1)) << 1) | (lane & (s - 1)));
-          const int hi = lo + s;
-          const bool up = ((lo & size) == 0);
-          const unsigned long long a = keys[lo], b = keys[hi];
-          if ((a > b) == up) { keys[lo] = b; keys[hi] = a; }
-        }
-        __syncwarp();
-      }
+    for (int base = warp * 64; base < sort_n; base += nwarps * 64) {
+      unsigned long long a = keys[base + lane], b = keys[base + 32 + lane];
+#pragma unroll
+      for (int s = 32; s > 0; s >>= 1) bitonic_step64(a, b, base, lane, s, size);
+      keys[base + lane] = a; keys[base + 32 + lane] = b;
     }
     __syncthreads();
   }
