@@ -38,6 +38,7 @@ constexpr int kMiscBytes = 1024 /*lse*/ + 3 * 256 * 8 /*merge*/;
 constexpr int kRawBytes = 2 * kMaxSegTiles * kTileKeys * 4;   // sweep 2: one partial-sum array per column half
 constexpr int kSmemBytes = 1024 /*align*/ + kQRegion + kKRegion + kMiscBytes + kRawBytes + 256 /*barriers*/;
 constexpr long long kDefaultWaitCycles = 4000000000ll;  // ~2 s: a wait that long is reported, not spun on
+constexpr uint32_t kSuspendNs = 4000;                   // a waiting thread sleeps in the barrier unit, not in a polling loop
 constexpr long long kDrainCycles = 2000000ll;           // ~1 ms: wait for own copies / MMAs in flight after an abort
 
 enum Mode { kNone = 0, kStats = 1, kEmit = 2 };
@@ -91,9 +92,9 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"     // may suspend the thread for up to the hint (ns)
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
   return ok != 0;
 }
 // Bounded wait: true once the barrier's phase is complete; gives up after `limit` clock ticks (false), records the failure (status[0] = the first wait site that
