@@ -40,11 +40,11 @@ NOMINAL_HBM_GBS = 8000.0
 # the kernel source they were measured on, for that per-layer shape and for four-layer groups only: any other
 # source hash, shape or grouping reports null.
 NCU_TRAFFIC = {
-    "kernel_sha256": "fbec4372a65a013bb9bac9081330579d55d3ffdec06bbf7f90f1e9fc13110969",
+    "kernel_sha256": "fd5486a528f4fa2725fa32204f75788ae948acc91e2776567469be5a1b045c41",
     "shape": (8, 128, 1, 32768, 32),          # Hkv, D, Bt, S, ws
     "layers_per_launch": 4,
-    "live_bytes_per_launch": 479_409_664 + 5_171_968,
-    "cold_bytes_per_launch": 541877248 + 7847424,
+    "live_bytes_per_launch": 475_897_344 + 5_187_072,
+    "cold_bytes_per_launch": 541769472 + 9059328,
 }
 
 
