@@ -40,11 +40,11 @@ NOMINAL_HBM_GBS = 8000.0
 # the kernel source they were measured on, for that per-layer shape and for four-layer groups only: any other
 # source hash, shape or grouping reports null.
 NCU_TRAFFIC = {
-    "kernel_sha256": "fd5486a528f4fa2725fa32204f75788ae948acc91e2776567469be5a1b045c41",
+    "kernel_sha256": "a25e0013ce5a5b0abf7384ba79ceacb14335fd780246ae05bfa1ce17c0f2121d",
     "shape": (8, 128, 1, 32768, 32),          # Hkv, D, Bt, S, ws
     "layers_per_launch": 4,
-    "live_bytes_per_launch": 475_897_344 + 5_187_072,
-    "cold_bytes_per_launch": 541769472 + 9059328,
+    "live_bytes_per_launch": 476_719_104 + 5_652_224,
+    "cold_bytes_per_launch": 541_775_360 + 7_707_392,
 }
 
 
