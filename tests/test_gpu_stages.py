@@ -96,6 +96,26 @@ def test_score_extreme_logits_do_not_overflow():
     U.assert_scores_close(got, ref, "extreme logits")
 
 
+def test_score_row_maximum_that_keeps_growing_along_the_prefix():
+    # Sweep 1 sums relative to a reference that it raises only when a chunk of keys turns out far above it.  Hot keys
+    # of growing strength in different tiles (and one beyond the last full tile) make every window row raise it
+    # several times in mid-stream, by tens to hundreds of powers of two; in between come keys far below it.
+    w = synth.Workload("grow", 18, L=1, Hq=4, Hkv=2, D=128, Bt=1, S=1500, ws=8, pool=3, N=4, Bl=8, m=1, recipe="iid")
+    t = synth.layer_inputs(w, 0)
+    q = synth.bf16_bits_to_f32(t["q"])
+    k = synth.bf16_bits_to_f32(t["k"])
+    for h in range(w.Hkv):
+        mean_q = q[0, h * w.G:(h + 1) * w.G].reshape(-1, w.D).mean(axis=0)
+        for pos, gain in ((40, 12.0), (300, 30.0), (301, -30.0), (700, 60.0), (1100, 5.0), (1400, 120.0)):
+            k[0, h, pos] = gain * mean_q
+    kb = synth.f32_to_bf16_bits(k)
+    with Ctx(w) as c:
+        got = gpu_scores(c, 0, t["q"], kb)
+    ref = O.window_scores(synth.bf16_bits_to_f64(t["q"]), synth.bf16_bits_to_f64(kb), w.ws, w.pool)["score"]
+    assert np.isfinite(got).all()
+    U.assert_scores_close(got, ref, "growing maximum")
+
+
 # ----------------------------------------------------------------------------------------- select
 def _inject(c: Ctx, layer, scores_f32):
     B.dkv_set_scores(c.h, layer, torch.from_numpy(scores_f32).cuda())
