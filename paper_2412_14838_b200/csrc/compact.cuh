@@ -29,13 +29,13 @@ gather_rows_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ v_
     const int row = row0 + j * rows_per_pass;
     if (row < n + ws) {
       const int from = row < n ? idx[(size_t)bh * idx_stride + row] : P + (row - n);
-      val[j] = src[(size_t)from * vec_per_row + c];
+      val[j] = __ldcs(&src[(size_t)from * vec_per_row + c]);      // read once: first in line for eviction from L2
     }
   }
 #pragma unroll
   for (int j = 0; j < kGatherRows; ++j) {
     const int row = row0 + j * rows_per_pass;
-    if (row < n + ws) dst[(size_t)row * vec_per_row + c] = val[j];
+    if (row < n + ws) __stcs(&dst[(size_t)row * vec_per_row + c], val[j]);
   }
 }
 

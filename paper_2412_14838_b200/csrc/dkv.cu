@@ -50,6 +50,7 @@ struct dkv_ctx {
   int pass_taper;       // group sizes halve towards the end of the pass
   int pass_group;       // layers per scoring launch of dkv_run_prefill_pass (1..tc::kMaxGroup)
   bool emit_backward;   // sweep 2 walks every CTA's slice from the end to the start
+  int retain_mb;        // MB of a sweep-1 job's keys (the end of every CTA's slice) marked to stay in L2 for sweep 2
   long long wait_cycles;   // limit of the scoring kernel's mbarrier waits (dkv_set_wait_limit)
   int withhold_sweep, withhold_tile;   // test hook of dkv_debug_withhold_tile (-1: off)
   float2* d_tc_stats;   // [3][kMaxGroup*Bt*Hkv][tc_slots][256]: partial softmax statistics, three jobs in rotation
@@ -221,6 +222,7 @@ bool make_job(dkv_ctx* c, int mode, int layer, int nl, const void* const* q, con
   p->S = s.S; p->P = s.P; p->ws = s.ws; p->M = s.M; p->D = s.D; p->heads = nl * heads; p->half = s.pool / 2;
   p->nl = nl; p->hpl = heads;
   p->back = (mode == tc::kEmit && c->emit_backward) ? 1 : 0;
+  p->retain_tiles = (int)((long long)c->retain_mb * (1 << 20) / ((long long)(c->tc_grid > 0 ? c->tc_grid : 1) * tc::kTileKeys * s.D * 2));
   p->wait_cycles = c->wait_cycles;
   p->withhold_tile = c->withhold_sweep == mode ? c->withhold_tile : -1;
   p->tph = (s.S + tc::kTileKeys - 1) / tc::kTileKeys;
@@ -587,6 +589,12 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
     c->pass_taper = env_int("DKV_PASS_TAPER", 0, 0, 1);
     c->n_side = env_int("DKV_SIDE_STREAMS", kSideStreams, 1, kSideStreams);
     c->emit_backward = env_int("DKV_EMIT_FORWARD", 0, 0, 1) == 0;
+    // Sweep 2 starts on the keys sweep 1 streamed last: that much of a job (4/7 of L2, 72 of 126 MB) is loaded with
+    // an evict-last policy, every other key tile and the gather's rows evict-first, so that neither the rest of the
+    // stream nor the side kernels' traffic pushes it out before it is read again.
+    int l2_bytes = 0;
+    if (cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, c->device) != cudaSuccess) l2_bytes = 0;
+    c->retain_mb = c->emit_backward ? env_int("DKV_L2_RETAIN_MB", (int)(((long long)l2_bytes * 4 / 7) >> 20), 0, 1024) : 0;
     c->wait_cycles = tc::kDefaultWaitCycles;
     c->withhold_sweep = c->withhold_tile = -1;
   }

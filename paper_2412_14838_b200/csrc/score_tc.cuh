@@ -65,6 +65,8 @@ struct Params {
   int back;                // sweep 2: 1 = every CTA walks its slice from the end to the start, so that it begins
                            // with the keys sweep 1 streamed last (those still in L2)
   long long wait_cycles;   // limit of every mbarrier wait, in clock64 ticks
+  int retain_tiles;        // sweep 1: the last `retain_tiles` key tiles of a CTA's slice are kept in L2 for sweep 2, which starts
+                           // with them; every other key tile of either sweep is marked to be evicted first (0: no marking)
   int withhold_tile;       // test hook: CTA 0 never loads its key tile number `withhold_tile` of this job (-1: off),
                            // so that the wait for it runs out and the timeout path can be exercised
 };
@@ -125,6 +127,23 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+// The same copy with an L2 eviction policy for the lines it brings in.
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -378,6 +397,8 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
         SegIter it(p, blockIdx.x, gridDim.x);
         Seg sg;
         int job_tile = 0;
+        const int keep_from = p.mode == kStats ? (int)(it.u_end - it.u) - p.retain_tiles : 0x7fffffff;
+        const uint64_t pol_first = l2_policy_evict_first(), pol_last = l2_policy_evict_last();
         while (ok && it.next(sg)) {
           const int hh = sg.bh % p.hpl;
           const CUtensorMap* q_map = &maps.q[sg.bh / p.hpl];
@@ -399,8 +420,14 @@ score_tc_kernel(const __grid_constant__ Maps maps0, const __grid_constant__ Maps
             if (!mbar_wait(EMPTY(s), (n & 1) ^ 1, abort_flag, p.status, 102, p.wait_cycles)) { ok = false; break; }
             if (job_tile == withhold) { withheld = tile; continue; }   // test hook: this tile never arrives
             mbar_expect_tx(FULL(s), tile_bytes);
-            for (int h = 0; h < halves; ++h)
-              tma_load_3d(smem_u32(k_smem + (s * 2 + h) * kHalfBytes), k_map, FULL(s), 64 * h, sg.key0 + i * kTileKeys, hh);
+            if (p.retain_tiles > 0) {
+              const uint64_t pol = job_tile >= keep_from ? pol_last : pol_first;
+              for (int h = 0; h < halves; ++h)
+                tma_load_3d_hint(smem_u32(k_smem + (s * 2 + h) * kHalfBytes), k_map, FULL(s), 64 * h, sg.key0 + i * kTileKeys, hh, pol);
+            } else {
+              for (int h = 0; h < halves; ++h)
+                tma_load_3d(smem_u32(k_smem + (s * 2 + h) * kHalfBytes), k_map, FULL(s), 64 * h, sg.key0 + i * kTileKeys, hh);
+            }
           }
         }
       }
