@@ -40,11 +40,11 @@ NOMINAL_HBM_GBS = 8000.0
 # the kernel source they were measured on, for that per-layer shape and for four-layer groups only: any other
 # source hash, shape or grouping reports null.
 NCU_TRAFFIC = {
-    "kernel_sha256": "a25e0013ce5a5b0abf7384ba79ceacb14335fd780246ae05bfa1ce17c0f2121d",
+    "kernel_sha256": "303acb3e0fa3bf64ba7b5cb1069bb408c1cc9088dab894f6a69887c302ea26de",
     "shape": (8, 128, 1, 32768, 32),          # Hkv, D, Bt, S, ws
     "layers_per_launch": 4,
-    "live_bytes_per_launch": 476_719_104 + 5_652_224,
-    "cold_bytes_per_launch": 541_775_360 + 7_707_392,
+    "live_bytes_per_launch": 478_000_384 + 28_855_296,
+    "cold_bytes_per_launch": 540_321_280 + 6_633_728,
 }
 
 
