@@ -412,11 +412,17 @@ def run_gpu(args, w):
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / e2e_steps
         dt = max_over_ranks(dt)
-        h2d = sum(t.numel() * 2 for t in hq) + sum(t.numel() * 2 for t in hk) + sum(t.numel() * 2 for t in hv)
-        # copied back: the counts and the valid rows (count + ws) of every head's K and V buffers
-        d2h = int((counts.astype(np.int64) + w.ws).sum()) * w.Hkv * w.D * 2 * 2 + counts.nbytes
+        # in: q and k in full and, of v, the rows the gather reads in place from the pinned buffers (count + ws per
+        # head at gather time); out: the counts and the valid rows of every head's K and V buffers.  The library
+        # counts them from the copies it issues and the rows it gathers; the full tensors are given beside them.
+        h2d, d2h = B.dkv_host_pass_bytes(ctx)
+        h2d_full = sum(t.numel() * 2 for t in hq) + sum(t.numel() * 2 for t in hk) + sum(t.numel() * 2 for t in hv)
+        assert d2h == int((counts.astype(np.int64) + w.ws).sum()) * w.Hkv * w.D * 2 * 2 + counts.nbytes
         e2e = {"value": whole_job_value(tokens, world, dt), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-               "ms_per_step": dt * 1e3, "steps": e2e_steps, "api": "dkv_run_prefill_pass_host (pinned host buffers)"}
+               "ms_per_step": dt * 1e3, "steps": e2e_steps, "api": "dkv_run_prefill_pass_host (pinned host buffers)",
+               "host_input_bytes": int(h2d_full),
+               "note": ("of V only the gathered rows cross the bus (read in place from pinned memory by the gather kernel)"
+                        if h2d < h2d_full else "q, k and v copied in full")}
 
     B.dkv_destroy(ctx)
     out = None

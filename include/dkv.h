@@ -197,13 +197,20 @@ int dkv_run_prefill_pass(dkv_ctx* ctx, const void* const* q_win, const void* con
 int dkv_run_prefill_pass_lse(dkv_ctx* ctx, const void* const* q_win, const void* const* k, const void* const* v,
                              const float* const* lse, void* const* kb, void* const* vb, void* stream);
 
-/* The same pass with all tensors in HOST memory (pinned memory recommended): each layer's q, k, v
- * are copied to device staging buffers owned by the context, processed, and after the last update
+/* The same pass with all tensors in HOST memory (pinned memory recommended): each layer's q and k
+ * are copied to device staging buffers owned by the context and processed; of v only the kept rows are
+ * needed (Algorithm 1 gathers V_c at the selected indices), so where v[l] is page-locked memory that
+ * kernels can address (cudaHostAlloc / cudaHostRegister) the gather reads those rows in place and the
+ * rest of v never crosses the bus; pageable v is copied in full like k.  After the last update
  * the counts and, of every layer's kb/vb, the valid rows of every head (count + ws; the rest of the
  * fixed-stride host buffers is left untouched) are copied back.  Synchronises.
  * q_win, k, v, kb, vb : host arrays of L HOST pointers; counts_out : host int32 [Bt, L]. */
 int dkv_run_prefill_pass_host(dkv_ctx* ctx, const void* const* q_win, const void* const* k,
                               const void* const* v, void* const* kb, void* const* vb, int32_t* counts_out);
+
+/* Bytes the last dkv_run_prefill_pass_host of this context moved: host to device (q, k, and v in full or
+ * its gathered rows) and device to host (counts and the valid rows of kb/vb).  h2d, d2h : host int64. */
+int dkv_host_pass_bytes(dkv_ctx* ctx, int64_t* h2d, int64_t* d2h);
 
 /* Fixed-pattern budgets: the per-layer schedules of the methods the paper compares with (Section 5.1,
  * "Baselines"), applied through the same select / compact kernels in place of Eq. 4-6.  Needs every layer

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(HERE, "libdkv.so")
 
 EXPORTS = [
     "dkv_create", "dkv_destroy", "dkv_reset", "dkv_score", "dkv_score_static", "dkv_score_lse", "dkv_set_scores", "dkv_select_topk", "dkv_rebudget",
-    "dkv_compact", "dkv_compact_all", "dkv_run_prefill_pass", "dkv_run_prefill_pass_lse", "dkv_run_prefill_pass_host",
+    "dkv_compact", "dkv_compact_all", "dkv_run_prefill_pass", "dkv_run_prefill_pass_lse", "dkv_run_prefill_pass_host", "dkv_host_pass_bytes",
     "dkv_apply_policy", "dkv_select_positions", "dkv_decode_attend", "dkv_get_counts",
     "dkv_layer_views", "dkv_kept_sorted", "dkv_budget_views", "dkv_memcpy_to_host", "dkv_last_status",
     "dkv_static_last_status", "dkv_set_wait_limit", "dkv_debug_withhold_tile", "dkv_profile", "dkv_profile_read", "dkv_launch_count", "dkv_last_cuda_error",
@@ -66,6 +66,7 @@ def load() -> ctypes.CDLL:
         "dkv_run_prefill_pass": [vp, pp, pp, pp, pp, pp, vp],
         "dkv_run_prefill_pass_host": [vp, pp, pp, pp, pp, pp, vp],
         "dkv_run_prefill_pass_lse": [vp, pp, pp, pp, pp, pp, pp, vp],
+        "dkv_host_pass_bytes": [vp, vp, vp],
         "dkv_apply_policy": [vp, i32, vp, vp],
         "dkv_select_positions": [vp, i32, i32, i32, vp],
         "dkv_decode_attend": [vp, i32, i32, i32, pp, pp, pp, pp, vp],
@@ -215,6 +216,13 @@ def dkv_run_prefill_pass_host(ctx: int, q_win: Sequence, k: Sequence, v: Sequenc
                               counts_out=None) -> None:
     _check(load().dkv_run_prefill_pass_host(ctx, _ptr_array(q_win), _ptr_array(k), _ptr_array(v), _ptr_array(kb),
                                             _ptr_array(vb), _ptr(counts_out)), "dkv_run_prefill_pass_host")
+
+
+def dkv_host_pass_bytes(ctx: int):
+    """(host-to-device, device-to-host) bytes moved by the context's last dkv_run_prefill_pass_host."""
+    h2d, d2h = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(load().dkv_host_pass_bytes(ctx, ctypes.byref(h2d), ctypes.byref(d2h)), "dkv_host_pass_bytes")
+    return int(h2d.value), int(d2h.value)
 
 
 def dkv_run_prefill_pass_lse(ctx: int, q_win: Sequence, k: Sequence, v: Sequence, lse: Sequence, kb: Sequence,

@@ -50,6 +50,8 @@ struct dkv_ctx {
   int pass_taper;       // group sizes halve towards the end of the pass
   int pass_group;       // layers per scoring launch of dkv_run_prefill_pass (1..tc::kMaxGroup)
   bool emit_backward;   // sweep 2 walks every CTA's slice from the end to the start
+  bool host_v_staged;   // dkv_run_prefill_pass_host copies V in full even where the gather could read its rows in place
+  long long host_h2d, host_d2h;   // bytes the last dkv_run_prefill_pass_host moved in either direction
   int retain_mb;        // MB of a sweep-1 job's keys (the end of every CTA's slice) marked to stay in L2 for sweep 2
   long long wait_cycles;   // limit of the scoring kernel's mbarrier waits (dkv_set_wait_limit)
   int withhold_sweep, withhold_tile;   // test hook of dkv_debug_withhold_tile (-1: off)
@@ -595,6 +597,8 @@ int dkv_create(const dkv_config* cfg, dkv_ctx** out) {
     int l2_bytes = 0;
     if (cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, c->device) != cudaSuccess) l2_bytes = 0;
     c->retain_mb = c->emit_backward ? env_int("DKV_L2_RETAIN_MB", (int)(((long long)l2_bytes * 4 / 7) >> 20), 0, 1024) : 0;
+    c->host_v_staged = env_int("DKV_HOST_V_STAGED", 0, 0, 1) != 0;
+    c->host_h2d = c->host_d2h = 0;
     c->wait_cycles = tc::kDefaultWaitCycles;
     c->withhold_sweep = c->withhold_tile = -1;
   }
@@ -827,17 +831,37 @@ int dkv_run_prefill_pass_host(dkv_ctx* c, const void* const* q_win, const void* 
   if (rc) return rc;
   cudaStream_t cp = c->st_copy, st = c->st_comp;
   if ((rc = do_reset(c, st))) return rc;
+  // Only the kept rows of V are ever needed on the device (count + ws of S per head).  Where the caller's V is
+  // page-locked host memory that kernels can address, the gather reads exactly those rows over the bus instead of
+  // V being copied in full first; pageable memory (or DKV_HOST_V_STAGED=1) takes the full copy.
+  const void* v_dev[DKV_MAX_LAYERS];
+  for (int l = 0; l < s.L; ++l) {
+    v_dev[l] = nullptr;
+    if (c->host_v_staged) continue;
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, v[l]) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer && aligned16(at.devicePointer))
+      v_dev[l] = at.devicePointer;
+    else
+      cudaGetLastError();                      // an unregistered pointer is not an error here
+  }
+  const long long row_bytes = (long long)s.D * 2;
+  long long h2d = 0;
   for (int l = 0; l < s.L; ++l) {
     const int slot = l & 1;
     if (l >= 2) DKV_CUDA(c, cudaStreamWaitEvent(cp, c->ev_consumed[slot], 0));
     DKV_CUDA(c, cudaMemcpyAsync(c->st_q[slot], q_win[l], layer_q_bytes(s), cudaMemcpyHostToDevice, cp));
     DKV_CUDA(c, cudaMemcpyAsync(c->st_k[slot], k[l], layer_kv_bytes(s), cudaMemcpyHostToDevice, cp));
-    DKV_CUDA(c, cudaMemcpyAsync(c->st_v[slot], v[l], layer_kv_bytes(s), cudaMemcpyHostToDevice, cp));
+    h2d += (long long)layer_q_bytes(s) + (long long)layer_kv_bytes(s);
+    if (!v_dev[l]) {
+      DKV_CUDA(c, cudaMemcpyAsync(c->st_v[slot], v[l], layer_kv_bytes(s), cudaMemcpyHostToDevice, cp));
+      h2d += (long long)layer_kv_bytes(s);
+    }
     DKV_CUDA(c, cudaEventRecord(c->ev_copied[slot], cp));
     DKV_CUDA(c, cudaStreamWaitEvent(st, c->ev_copied[slot], 0));
     if ((rc = do_score(c, l, c->st_q[slot], c->st_k[slot], nullptr, st))) return rc;
     if ((rc = do_select(c, l, nullptr, nullptr, st))) return rc;
-    if ((rc = do_gather(c, l, c->st_k[slot], c->st_v[slot], c->st_kb[l], c->st_vb[l], st))) return rc;
+    if ((rc = do_gather(c, l, c->st_k[slot], v_dev[l] ? v_dev[l] : c->st_v[slot], c->st_kb[l], c->st_vb[l], st))) return rc;
+    if (v_dev[l]) h2d += (long long)(c->sel_n[l] + s.ws) * s.Bt * s.Hkv * row_bytes;
     DKV_CUDA(c, cudaEventRecord(c->ev_consumed[slot], st));
     const bool update = ((l + 1) % s.m == 0) || (l + 1 == s.L && s.L % s.m != 0);
     if (update) {
@@ -862,8 +886,17 @@ int dkv_run_prefill_pass_host(dkv_ctx* c, const void* const* q_win, const void* 
                                     cudaMemcpyDeviceToHost, st));
     }
   if (counts_out) memcpy(counts_out, counts.data(), sizeof(int) * s.Bt * s.L);
+  long long d2h = (long long)sizeof(int) * s.Bt * s.L;
+  for (size_t i = 0; i < counts.size(); ++i) d2h += 2ll * (counts[i] + s.ws) * s.Hkv * row_bytes;
+  c->host_h2d = h2d; c->host_d2h = d2h;
   DKV_CUDA(c, cudaStreamSynchronize(cp));
   DKV_CUDA(c, cudaStreamSynchronize(st));
+  return DKV_OK;
+}
+
+int dkv_host_pass_bytes(dkv_ctx* c, int64_t* h2d, int64_t* d2h) {
+  if (!c || !h2d || !d2h) return DKV_ERR_INVALID_ARG;
+  *h2d = c->host_h2d; *d2h = c->host_d2h;
   return DKV_OK;
 }
 

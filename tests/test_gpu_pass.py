@@ -372,13 +372,22 @@ def test_host_buffer_pass_matches_device_pass():
         okb = [torch.zeros(shape, dtype=torch.int16).pin_memory() for _ in range(w.L)]
         ovb = [torch.zeros(shape, dtype=torch.int16).pin_memory() for _ in range(w.L)]
         counts = np.zeros((w.Bt, w.L), dtype=np.int32)
-        for _ in range(2):                              # the second call reuses the staging buffers
-            B.dkv_run_prefill_pass_host(g.h, hq, hk, hv, okb, ovb, counts)
-            assert (counts == g.counts).all()
-            for l in range(w.L):
-                n = int(counts[0, l]) + w.ws
-                assert torch.equal(okb[l][:, :, :n], g.kb[l].cpu()[:, :, :n])
-                assert torch.equal(ovb[l][:, :, :n], g.vb[l].cpu()[:, :, :n])
+        full = sum(t.numel() * 2 for t in hq + hk + hv)
+        rows_in_place = w.L * (w.Blc + w.ws) * w.Bt * w.Hkv * w.D * 2
+        # pinned V: the gather reads its rows in place; pageable V (a plain numpy array): copied in full
+        for hv_, h2d_want in ((hv, full - sum(t.numel() * 2 for t in hv) + rows_in_place), ([t["v"] for t in g.host], full)):
+            for _ in range(2):                          # the second call reuses the staging buffers
+                for o in okb + ovb:
+                    o.zero_()
+                B.dkv_run_prefill_pass_host(g.h, hq, hk, hv_, okb, ovb, counts)
+                assert (counts == g.counts).all()
+                for l in range(w.L):
+                    n = int(counts[0, l]) + w.ws
+                    assert torch.equal(okb[l][:, :, :n], g.kb[l].cpu()[:, :, :n])
+                    assert torch.equal(ovb[l][:, :, :n], g.vb[l].cpu()[:, :, :n])
+                h2d, d2h = B.dkv_host_pass_bytes(g.h)
+                assert h2d == h2d_want
+                assert d2h == int((counts.astype(np.int64) + w.ws).sum()) * w.Hkv * w.D * 2 * 2 + counts.nbytes
     finally:
         g.close()
 
