@@ -71,18 +71,20 @@ __device__ __forceinline__ void find_digit(const unsigned int* hist, int nbins, 
   __syncthreads();
 }
 
-// Warp-aggregated counter bump: lanes with equal `digit` share one atomicAdd.  Inactive lanes pass
-// active = false.  Returns, for active lanes, a distinct slot: old counter value + rank inside the group.
-// Must be called by all 32 lanes.
-__device__ __forceinline__ unsigned int agg_bump(unsigned int* counters, unsigned int digit, bool active) {
+// Counter bump without a return value for digits that come in runs (pooled scores: neighbouring positions share
+// their digit): a run of equal digits in adjacent lanes makes one atomicAdd of its length.  Equal digits that are
+// not adjacent are added separately.  Must be called by all 32 lanes.
+__device__ __forceinline__ void run_bump(unsigned int* counters, unsigned int digit, bool active) {
   const unsigned int lane = threadIdx.x & 31;
   const unsigned int key = active ? digit : 0xFFFFFFFFu;
-  const unsigned int peers = __match_any_sync(0xFFFFFFFFu, key);
-  const int leader = __ffs(peers) - 1;
-  unsigned int base = 0;
-  if (active && (int)lane == leader) base = atomicAdd(&counters[digit], (unsigned int)__popc(peers));
-  base = __shfl_sync(0xFFFFFFFFu, base, leader);
-  return base + (unsigned int)__popc(peers & ((1u << lane) - 1u));
+  const unsigned int prev = __shfl_up_sync(0xFFFFFFFFu, key, 1);
+  const bool head = lane == 0 || prev != key;
+  const unsigned int heads = __ballot_sync(0xFFFFFFFFu, head);
+  if (head && active) {
+    const unsigned int later = heads & ~((2u << lane) - 1u);       // run heads after this lane (lane 31: none)
+    const int next = later ? __ffs(later) - 1 : 32;
+    atomicAdd(&counters[digit], (unsigned int)(next - (int)lane));
+  }
 }
 
 // One compare-exchange step of a bitonic network on the 64 keys a warp holds in registers: lane j has
@@ -195,7 +197,7 @@ select_topk_kernel(const float* __restrict__ scores, int* __restrict__ idx, int*
   // pass 0: first digit of every score; neighbours share digits after pooling, so lanes combine their bumps
   for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
   __syncthreads();
-  DKV_SEL_FOR(e) agg_bump(hist, val(e) >> 21, DKV_SEL_OK(e));
+  DKV_SEL_FOR(e) run_bump(hist, val(e) >> 21, DKV_SEL_OK(e));
   __syncthreads();
   {
     unsigned int* gh = layer_hist + (size_t)(blockIdx.x / Hkv) * kBins;
